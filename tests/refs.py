@@ -1,0 +1,111 @@
+"""Independent reference computations used to pin the CPU oracle.
+
+Nothing here is derived from the oracle's code: ``brute_force`` is the
+definition of a CTC labelling probability (sum over all alignments that
+collapse to the labelling), ``PyPrefixSearch`` is a second, separately
+written dictionary-of-tuples prefix beam search, ``greedy`` is best-path
+decoding.
+"""
+from __future__ import annotations
+
+import itertools
+import math
+
+import numpy as np
+
+
+def collapse(path, blank):
+    out, prev = [], None
+    for c in path:
+        if c != prev and c != blank:
+            out.append(int(c))
+        prev = c
+    return tuple(out)
+
+
+def brute_force(lp: np.ndarray, blank: int, keep: np.ndarray | None = None) -> dict:
+    """log P(labelling) for every labelling, by enumerating all V**T alignments.
+
+    ``keep`` [T,V] (bool) restricts each frame to its surviving tokens.
+    Probabilities are summed in float64 with math.fsum.
+    """
+    T, V = lp.shape
+    terms: dict = {}
+    p = np.exp(lp.astype(np.float64))
+    for path in itertools.product(range(V), repeat=T):
+        if keep is not None and not all(keep[t, c] for t, c in enumerate(path)):
+            continue
+        w = 1.0
+        for t, c in enumerate(path):
+            w *= p[t, c]
+        terms.setdefault(collapse(path, blank), []).append(w)
+    return {k: (math.log(s) if (s := math.fsum(v)) > 0 else -math.inf) for k, v in terms.items()}
+
+
+def greedy(lp: np.ndarray, blank: int):
+    return collapse(lp.argmax(axis=1).tolist(), blank)
+
+
+def _lse(a, b):
+    if a == -math.inf:
+        return b
+    if b == -math.inf:
+        return a
+    m = max(a, b)
+    return m + math.log1p(math.exp(min(a, b) - m))
+
+
+class PyPrefixSearch:
+    """Dictionary-keyed CTC prefix beam search, optional per-frame survivor sets."""
+
+    def __init__(self, blank: int, K: int):
+        self.blank, self.K = blank, K
+        self.beam = {(): (0.0, -math.inf)}
+        self.revivals = 0          # prefixes that re-entered the beam after leaving it
+        self._ever = {()}
+        self._prev = {()}
+
+    def step(self, lp_row, survivors):
+        nxt: dict = {}
+
+        def add(key, which, val):
+            pb, pnb = nxt.get(key, (-math.inf, -math.inf))
+            nxt[key] = (_lse(pb, val), pnb) if which == 0 else (pb, _lse(pnb, val))
+
+        for seq, (pb, pnb) in self.beam.items():
+            tot = _lse(pb, pnb)
+            for c in survivors:
+                v = float(lp_row[c])
+                if c == self.blank:
+                    add(seq, 0, tot + v)
+                elif seq and c == seq[-1]:
+                    add(seq, 1, pnb + v)
+                    add(seq + (c,), 1, pb + v)
+                else:
+                    add(seq + (c,), 1, tot + v)
+        items = [(k, v) for k, v in nxt.items() if _lse(*v) > -math.inf]
+        items.sort(key=lambda kv: (-_lse(*kv[1]), len(kv[0]), kv[0]))
+        self.beam = dict(items[: self.K])
+        now = set(self.beam)
+        self.revivals += len([s for s in now if s in self._ever and s not in self._prev])
+        self._ever |= now
+        self._prev = now
+
+    def results(self):
+        out = [(k, _lse(*v)) for k, v in self.beam.items()]
+        out.sort(key=lambda kv: (-kv[1], len(kv[0]), kv[0]))
+        return out
+
+
+def py_decode(lp: np.ndarray, blank: int, K: int, log_r: np.float32 | None):
+    """Decode one utterance [T,V]; ``log_r`` None means no survivor test at all."""
+    T, V = lp.shape
+    s = PyPrefixSearch(blank, K)
+    for t in range(T):
+        if log_r is None:
+            surv = range(V)
+        else:
+            thr = np.float32(lp[t].max()) + np.float32(log_r)
+            surv = [c for c in range(V) if lp[t, c] >= thr]
+        s.step(lp[t], surv)
+    return s
