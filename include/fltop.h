@@ -1,0 +1,150 @@
+/*
+ * fltop.h - C ABI of the frame-pruned CTC prefix beam search library (sm_100a).
+ *
+ * The library decodes frame-level log-probability emissions with the
+ * procedure of the FLToP CTC paper (Algorithm 1): the beam starts with the
+ * empty prefix; at every frame only tokens whose probability is at least R
+ * times the frame's top probability extend the beam (the conditional break of
+ * Algorithm 1, Section 3); candidates naming the same prefix are combined and
+ * the best beam_size are kept (SelectTopK); after the last frame the
+ * hypotheses are returned best first (GetHighestScorePrefix, widened to the
+ * whole beam).  The CTC collapsing rule is the standard one of the "standard
+ * BeamSearchCTC decoders" the paper modifies (Section 3): each prefix carries
+ * the log-mass of alignments ending in blank and ending in its last token.
+ * The top-N stage, beam_threshold and the language model of Algorithm 1 are
+ * not implemented (their config fields are reserved).
+ *
+ * Conventions
+ *   - every `d_*` pointer is DEVICE memory owned by the caller; the library
+ *     never frees or keeps it beyond the call's work on `cuda_stream`.
+ *   - calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream) and return without synchronising;
+ *     outputs are valid once the caller has synchronised the stream.
+ *   - the return value reports what the host can detect (bad arguments,
+ *     capacity of the handle, CUDA launch errors).  Conditions only the
+ *     device sees are reported per utterance in `d_status`.
+ *   - no call prints, throws or aborts.  A handle must not be used from two
+ *     threads at once; distinct handles are independent.
+ */
+#ifndef FLTOP_H_
+#define FLTOP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fltop_handle fltop_handle; /* opaque, owned by the library */
+
+enum {
+  FLTOP_OK = 0,
+  FLTOP_ERR_INVALID_ARG = 1, /* null pointer, value out of range, reserved field set */
+  FLTOP_ERR_CUDA = 2,        /* a CUDA runtime call failed (see fltop_last_cuda_error) */
+  FLTOP_ERR_OOM = 3,         /* workspace allocation failed or caller workspace too small */
+  FLTOP_ERR_CAPACITY = 4,    /* B, T, S or C above what the handle was created for; per
+                                utterance: trie arena full or output length above max_out_len */
+  FLTOP_ERR_STATE = 5        /* call not valid for this handle (decode on a streaming
+                                handle or the reverse) */
+};
+
+/* Per-utterance device status bits written to d_status (0 = fine). */
+enum {
+  FLTOP_ST_BAD_LENGTH = 1,   /* length < 0 or > T: utterance skipped, nhyp = 0 */
+  FLTOP_ST_ARENA_FULL = 2,   /* prefix trie arena exhausted: results of this utterance invalid */
+  FLTOP_ST_TRUNCATED = 4,    /* a hypothesis is longer than max_out_len: tokens cut, lens true */
+  FLTOP_ST_EMPTY_BEAM = 8,   /* every candidate had probability 0 (all -inf rows) */
+  FLTOP_ST_INTERNAL = 16     /* a bounded device loop gave up; results invalid */
+};
+
+typedef struct {
+  int32_t vocab_size;     /* V, 2 <= V <= 8192 */
+  int32_t blank_id;       /* 0 <= blank_id < V */
+  int32_t beam_width;     /* K = beam_size of Algorithm 1, 1 <= K <= 2048 */
+  float threshold_r;      /* R of Algorithm 1 in the probability domain, 0 <= R <= 1;
+                             0 disables pruning.  A token survives a frame iff
+                             logp >= logp_max + (float)log((double)R), float32 compare */
+  int32_t max_batch;      /* capacity: utterances per fltop_decode call / concurrent streams */
+  int32_t max_frames;     /* capacity: frames per utterance (decode) or per stream between
+                             two resets (stream_step) */
+  int32_t max_chunk_frames; /* 0: the handle serves fltop_decode.  > 0: the handle serves
+                             fltop_stream_step with chunks of at most this many frames */
+  int32_t max_out_len;    /* L of the token output, 1 <= L */
+  int32_t top_n;          /* reserved (N of Algorithm 1); must be 0 */
+  float beam_threshold;   /* reserved (beam_threshold of Algorithm 1); must be <= 0 */
+  int32_t device;         /* CUDA device ordinal */
+  void* workspace;        /* optional DEVICE memory, 256-byte aligned, for all of the
+                             handle's scratch; NULL = the library allocates it */
+  size_t workspace_bytes; /* size of `workspace`; ignored when workspace is NULL */
+} fltop_config;
+
+/* Bytes of device scratch a handle with this config needs (0 on invalid config). */
+size_t fltop_workspace_size(const fltop_config* cfg);
+
+/* Algorithm 1, procedure header: fixes beam_size, R and the shapes.  Validates cfg,
+ * sizes and allocates (or adopts) the workspace.  On success *out is a new handle. */
+int fltop_create(const fltop_config* cfg, fltop_handle** out);
+
+/* Algorithm 1 for a whole batch.  Each of the B utterances is decoded independently.
+ *   d_logp      [B,T,V] float32 log-probabilities; element strides stride_b, stride_t, the
+ *               V entries of a frame contiguous and 16-byte aligned when V % 4 == 0.
+ *               Frames t >= d_lengths[b] are never read.
+ *   d_lengths   [B] int32 frame counts.
+ *   d_tokens    [B,K,L] int32: hypothesis k of utterance b, L = max_out_len; entries past
+ *               the hypothesis' length are left untouched.
+ *   d_lens      [B,K] int32 true lengths (0 for unused slots k >= nhyp).
+ *   d_scores    [B,K] float32 log-probability of each hypothesis (log-sum of its blank and
+ *               non-blank mass at the last frame; -inf for unused slots); best first.
+ *   d_nhyp      [B] int32 number of hypotheses (<= K; 1 with the empty sequence and score 0
+ *               when the length is 0).
+ *   d_status    [B] int32 FLTOP_ST_* bits, may be NULL. */
+int fltop_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+                 const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_tokens,
+                 int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
+                 void* cuda_stream);
+
+/* Algorithm 1 consumed chunk by chunk: the frame loop of S concurrent streams advances by
+ * up to C frames; the beam of every stream is kept in the handle between calls.
+ *   d_chunk      [S,C,V] float32, contiguous.
+ *   d_chunk_lens [S] int32 valid frames of each stream in this chunk (0 = idle).
+ *   d_flags      [S] uint8, may be NULL: bit0 = reset the stream to the empty prefix before
+ *                consuming the chunk; bit1 = write this stream's current hypotheses.
+ *                NULL means "no reset, write hypotheses if output pointers are given".
+ *                A stream must be reset before its first chunk.
+ *   outputs as in fltop_decode with B = S; all four may be NULL together (no readback). */
+int fltop_stream_step(fltop_handle* h, const float* d_chunk, const int32_t* d_chunk_lens,
+                      const uint8_t* d_flags, int32_t S, int32_t C, int32_t* d_tokens,
+                      int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
+                      void* cuda_stream);
+
+/* Releases the handle and the workspace if the library allocated it. */
+int fltop_destroy(fltop_handle* h);
+
+/* The frame-level pruning step alone (Algorithm 1, conditional break), exactly as the two
+ * calls above run it: for every frame the survivors in ascending token order.
+ *   d_counts  [B,T] int32 survivors per frame (0 for frames past the length).
+ *   d_entries [B,T,V] pairs {int32 token, float32 logp}; the first d_counts[b,t] pairs of
+ *             frame (b,t) are valid. */
+int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+                const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_counts,
+                void* d_entries, void* cuda_stream);
+
+/* Optional helpers. */
+const char* fltop_status_string(int code);
+/* Last cudaError_t seen by this handle (0 if none). */
+int fltop_last_cuda_error(const fltop_handle* h);
+/* Bytes of beam state the handle holds: prefix trie arenas, stream states, survivor lists. */
+size_t fltop_beam_state_bytes(const fltop_handle* h);
+/* Kernels launched by this handle since creation. */
+int64_t fltop_launch_count(const fltop_handle* h);
+/* With profiling enabled every call brackets its kernels with CUDA events on the caller's
+ * stream.  fltop_last_kernel_ms synchronises on those events and returns the device time
+ * of the most recent call's {prune, decode} kernels in out_ms[0..1] (milliseconds). */
+int fltop_set_profiling(fltop_handle* h, int enable);
+int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLTOP_H_ */

@@ -1,0 +1,317 @@
+// Host side of the C ABI declared in include/fltop.h: argument validation,
+// workspace carve-up and kernel launches on the caller's stream.
+#include <cmath>
+#include <limits>
+#include <new>
+
+#include "../../include/fltop.h"
+#include "fltop_internal.h"
+
+using namespace fltop;
+
+struct fltop_handle {
+  fltop_config cfg;
+  float log_r;
+  bool owns_workspace;
+  unsigned char* ws;
+  size_t ws_bytes;
+  // regions of the workspace
+  int32_t* counts;
+  Survivor* entries;
+  TrieNode* nodes;
+  int32_t* state;
+  int64_t frame_cap;      // frames per utterance the survivor buffers hold
+  int64_t nodes_per_utt;
+  size_t beam_state_bytes;
+  int last_cuda;
+  int64_t launches;
+  bool profiling;
+  bool prof_valid;
+  cudaEvent_t ev[3];
+};
+
+namespace {
+
+constexpr size_t kMaxSmem = 227 * 1024;
+constexpr size_t kAlign = 256;
+
+size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+bool config_ok(const fltop_config* c) {
+  if (!c) return false;
+  if (c->vocab_size < 2 || c->vocab_size > 8192) return false;
+  if (c->blank_id < 0 || c->blank_id >= c->vocab_size) return false;
+  if (c->beam_width < 1 || c->beam_width > 2048) return false;
+  if (!(c->threshold_r >= 0.f && c->threshold_r <= 1.f)) return false;  // rejects NaN too
+  if (c->max_batch < 1 || c->max_frames < 1 || c->max_out_len < 1) return false;
+  if (c->max_chunk_frames < 0 || c->max_chunk_frames > c->max_frames) return false;
+  if (c->top_n != 0) return false;
+  if (c->beam_threshold > 0.f || c->beam_threshold != c->beam_threshold) return false;
+  if (c->device < 0) return false;
+  if ((int64_t)c->beam_width * c->max_frames + 1 > (int64_t)std::numeric_limits<int32_t>::max())
+    return false;
+  if (decode_smem_bytes(c->beam_width, c->vocab_size) > kMaxSmem) return false;
+  if (c->workspace && (reinterpret_cast<uintptr_t>(c->workspace) % kAlign) != 0) return false;
+  return true;
+}
+
+struct Layout {
+  size_t counts, entries, nodes, state, total, beam_state;
+  int64_t frame_cap, nodes_per_utt;
+};
+
+Layout layout_of(const fltop_config& c) {
+  Layout l;
+  l.frame_cap = c.max_chunk_frames > 0 ? c.max_chunk_frames : c.max_frames;
+  l.nodes_per_utt = (int64_t)c.beam_width * c.max_frames + 1;
+  const size_t frames = (size_t)c.max_batch * (size_t)l.frame_cap;
+  size_t off = 0;
+  l.counts = off; off += up(frames * sizeof(int32_t));
+  l.entries = off; off += up(frames * (size_t)c.vocab_size * sizeof(Survivor));
+  l.nodes = off; off += up((size_t)c.max_batch * (size_t)l.nodes_per_utt * sizeof(TrieNode));
+  l.state = off;
+  if (c.max_chunk_frames > 0) off += up((size_t)c.max_batch * state_words(c.beam_width) * 4);
+  l.total = off;
+  l.beam_state = off;  // survivor lists + trie arenas + stream states
+  return l;
+}
+
+int cuda_fail(fltop_handle* h, cudaError_t e) {
+  if (h) h->last_cuda = (int)e;
+  cudaGetLastError();  // clear the sticky-free error state
+  return FLTOP_ERR_CUDA;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool changed = false;
+  cudaError_t enter(int dev) {
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e != cudaSuccess) return e;
+    if (prev != dev) {
+      e = cudaSetDevice(dev);
+      changed = (e == cudaSuccess);
+    }
+    return e;
+  }
+  ~DeviceGuard() {
+    if (changed) cudaSetDevice(prev);
+  }
+};
+
+int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+               const int32_t* d_lengths, const uint8_t* d_flags, int32_t B, int32_t T,
+               bool streaming, int32_t* d_tokens, int32_t* d_lens, float* d_scores,
+               int32_t* d_nhyp, int32_t* d_status, cudaStream_t s) {
+  DeviceGuard g;
+  cudaError_t e = g.enter(h->cfg.device);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  h->prof_valid = false;
+  if (B == 0) return FLTOP_OK;
+
+  PruneParams pp;
+  pp.logp = d_logp; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
+  pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
+  pp.counts = h->counts; pp.entries = h->entries;
+
+  DecodeParams dp;
+  dp.lengths = d_lengths; dp.flags = d_flags; dp.B = B; dp.T = T; dp.V = h->cfg.vocab_size;
+  dp.K = h->cfg.beam_width; dp.blank = h->cfg.blank_id; dp.L = h->cfg.max_out_len;
+  dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
+  dp.counts = h->counts; dp.entries = h->entries; dp.nodes = h->nodes;
+  dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
+  dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
+  dp.out_status = d_status;
+
+  if (h->profiling) cudaEventRecord(h->ev[0], s);
+  if (T > 0) {
+    e = launch_prune(pp, s);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    ++h->launches;
+  }
+  if (h->profiling) cudaEventRecord(h->ev[1], s);
+  e = launch_decode(dp, s);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  ++h->launches;
+  if (h->profiling) {
+    cudaEventRecord(h->ev[2], s);
+    h->prof_valid = true;
+  }
+  return FLTOP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t fltop_workspace_size(const fltop_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return layout_of(*cfg).total;
+}
+
+int fltop_create(const fltop_config* cfg, fltop_handle** out) {
+  if (!out) return FLTOP_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(cfg)) return FLTOP_ERR_INVALID_ARG;
+  const Layout l = layout_of(*cfg);
+  if (cfg->workspace && cfg->workspace_bytes < l.total) return FLTOP_ERR_OOM;
+
+  int n_dev = 0;
+  cudaError_t e = cudaGetDeviceCount(&n_dev);
+  if (e != cudaSuccess) { cudaGetLastError(); return FLTOP_ERR_CUDA; }
+  if (cfg->device >= n_dev) return FLTOP_ERR_INVALID_ARG;
+  DeviceGuard g;
+  e = g.enter(cfg->device);
+  if (e != cudaSuccess) { cudaGetLastError(); return FLTOP_ERR_CUDA; }
+
+  fltop_handle* h = new (std::nothrow) fltop_handle();
+  if (!h) return FLTOP_ERR_OOM;
+  h->cfg = *cfg;
+  h->log_r = cfg->threshold_r > 0.f ? (float)std::log((double)cfg->threshold_r)
+                                    : -std::numeric_limits<float>::infinity();
+  h->last_cuda = 0; h->launches = 0; h->profiling = false; h->prof_valid = false;
+  h->ev[0] = h->ev[1] = h->ev[2] = nullptr;
+  if (cfg->workspace) {
+    h->ws = static_cast<unsigned char*>(cfg->workspace);
+    h->owns_workspace = false;
+  } else {
+    void* ptr = nullptr;
+    e = cudaMalloc(&ptr, l.total);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      delete h;
+      return e == cudaErrorMemoryAllocation ? FLTOP_ERR_OOM : FLTOP_ERR_CUDA;
+    }
+    h->ws = static_cast<unsigned char*>(ptr);
+    h->owns_workspace = true;
+  }
+  h->ws_bytes = l.total;
+  h->counts = reinterpret_cast<int32_t*>(h->ws + l.counts);
+  h->entries = reinterpret_cast<Survivor*>(h->ws + l.entries);
+  h->nodes = reinterpret_cast<TrieNode*>(h->ws + l.nodes);
+  h->state = cfg->max_chunk_frames > 0 ? reinterpret_cast<int32_t*>(h->ws + l.state) : nullptr;
+  h->frame_cap = l.frame_cap;
+  h->nodes_per_utt = l.nodes_per_utt;
+  h->beam_state_bytes = l.beam_state;
+  e = decode_prepare(cfg->beam_width, cfg->vocab_size);
+  if (e == cudaSuccess && h->state) {
+    // an un-reset stream holds an empty beam rather than garbage
+    e = cudaMemset(h->state, 0, (size_t)cfg->max_batch * state_words(cfg->beam_width) * 4);
+  }
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    if (h->owns_workspace) cudaFree(h->ws);
+    delete h;
+    return FLTOP_ERR_CUDA;
+  }
+  *out = h;
+  return FLTOP_OK;
+}
+
+int fltop_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+                 const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_tokens,
+                 int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
+                 void* cuda_stream) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  if (h->cfg.max_chunk_frames > 0) return FLTOP_ERR_STATE;
+  if (B < 0 || T < 0) return FLTOP_ERR_INVALID_ARG;
+  if (B > h->cfg.max_batch || T > h->cfg.max_frames) return FLTOP_ERR_CAPACITY;
+  if (B > 0 && (!d_lengths || !d_tokens || !d_lens || !d_scores || !d_nhyp))
+    return FLTOP_ERR_INVALID_ARG;
+  if (B > 0 && T > 0 && (!d_logp || stride_t < h->cfg.vocab_size || stride_b < 0))
+    return FLTOP_ERR_INVALID_ARG;
+  return run_decode(h, d_logp, stride_b, stride_t, d_lengths, nullptr, B, T, false, d_tokens,
+                    d_lens, d_scores, d_nhyp, d_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int fltop_stream_step(fltop_handle* h, const float* d_chunk, const int32_t* d_chunk_lens,
+                      const uint8_t* d_flags, int32_t S, int32_t C, int32_t* d_tokens,
+                      int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
+                      void* cuda_stream) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  if (h->cfg.max_chunk_frames <= 0) return FLTOP_ERR_STATE;
+  if (S < 0 || C < 0) return FLTOP_ERR_INVALID_ARG;
+  if (S > h->cfg.max_batch || C > h->cfg.max_chunk_frames) return FLTOP_ERR_CAPACITY;
+  if (S > 0 && !d_chunk_lens) return FLTOP_ERR_INVALID_ARG;
+  if (S > 0 && C > 0 && !d_chunk) return FLTOP_ERR_INVALID_ARG;
+  const int n_out = (d_tokens ? 1 : 0) + (d_lens ? 1 : 0) + (d_scores ? 1 : 0) + (d_nhyp ? 1 : 0);
+  if (n_out != 0 && n_out != 4) return FLTOP_ERR_INVALID_ARG;
+  const int64_t V = h->cfg.vocab_size;
+  return run_decode(h, d_chunk, (int64_t)C * V, V, d_chunk_lens, d_flags, S, C, true, d_tokens,
+                    d_lens, d_scores, d_nhyp, d_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+                const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_counts,
+                void* d_entries, void* cuda_stream) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  if (B < 0 || T < 0) return FLTOP_ERR_INVALID_ARG;
+  if (B == 0 || T == 0) return FLTOP_OK;
+  if (!d_logp || !d_lengths || !d_counts || !d_entries) return FLTOP_ERR_INVALID_ARG;
+  if (stride_t < h->cfg.vocab_size || stride_b < 0) return FLTOP_ERR_INVALID_ARG;
+  DeviceGuard g;
+  cudaError_t e = g.enter(h->cfg.device);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  PruneParams pp;
+  pp.logp = d_logp; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
+  pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
+  pp.counts = d_counts; pp.entries = static_cast<Survivor*>(d_entries);
+  e = launch_prune(pp, static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  ++h->launches;
+  return FLTOP_OK;
+}
+
+int fltop_destroy(fltop_handle* h) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  int rc = FLTOP_OK;
+  DeviceGuard g;
+  if (g.enter(h->cfg.device) != cudaSuccess) rc = FLTOP_ERR_CUDA;
+  for (int i = 0; i < 3; ++i)
+    if (h->ev[i]) cudaEventDestroy(h->ev[i]);
+  if (h->owns_workspace && h->ws && cudaFree(h->ws) != cudaSuccess) rc = FLTOP_ERR_CUDA;
+  cudaGetLastError();
+  delete h;
+  return rc;
+}
+
+const char* fltop_status_string(int code) {
+  switch (code) {
+    case FLTOP_OK: return "ok";
+    case FLTOP_ERR_INVALID_ARG: return "invalid argument";
+    case FLTOP_ERR_CUDA: return "CUDA runtime error";
+    case FLTOP_ERR_OOM: return "out of device memory or workspace too small";
+    case FLTOP_ERR_CAPACITY: return "request exceeds the handle's capacity";
+    case FLTOP_ERR_STATE: return "call not valid for this handle";
+    default: return "unknown status";
+  }
+}
+
+int fltop_last_cuda_error(const fltop_handle* h) { return h ? h->last_cuda : 0; }
+size_t fltop_beam_state_bytes(const fltop_handle* h) { return h ? h->beam_state_bytes : 0; }
+int64_t fltop_launch_count(const fltop_handle* h) { return h ? h->launches : 0; }
+
+int fltop_set_profiling(fltop_handle* h, int enable) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  if (enable && !h->ev[0]) {
+    DeviceGuard g;
+    cudaError_t e = g.enter(h->cfg.device);
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaEventCreate(&h->ev[i]);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+  }
+  h->profiling = enable != 0;
+  h->prof_valid = false;
+  return FLTOP_OK;
+}
+
+int fltop_last_kernel_ms(fltop_handle* h, float* out_ms) {
+  if (!h || !out_ms) return FLTOP_ERR_INVALID_ARG;
+  if (!h->profiling || !h->prof_valid) return FLTOP_ERR_STATE;
+  cudaError_t e = cudaEventSynchronize(h->ev[2]);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&out_ms[0], h->ev[0], h->ev[1]);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&out_ms[1], h->ev[1], h->ev[2]);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  return FLTOP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,78 @@
+// Internal declarations shared by the CUDA translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace fltop {
+
+// One survivor of a frame: token id and its float32 log-probability.
+struct __align__(8) Survivor {
+  int32_t token;
+  float logp;
+};
+
+// Prefix-trie node (one per distinct prefix of an utterance, 32 bytes).
+// Children of a node form a singly linked list (first_child / next_sibling);
+// child_filter has bit (token & 63) set for every child ever created, so that
+// "no such child yet" is decided without touching the list.
+struct __align__(32) TrieNode {
+  int32_t parent;        // node id of the prefix without its last token, -1 for the root
+  int32_t token;         // last token of the prefix, -1 for the root
+  int32_t first_child;   // head of the child list, -1 if none
+  int32_t next_sibling;  // next child of `parent`, -1 at the end
+  int32_t depth;         // number of tokens
+  int32_t pad;
+  unsigned long long child_filter;
+};
+
+// Per-stream state header kept in HBM between stream_step calls.
+struct StateHeader {
+  int32_t nbeam;      // live beam entries
+  int32_t n_nodes;    // trie nodes allocated (node 0 = empty prefix)
+  int32_t frames;     // frames consumed since the last reset
+  int32_t status;     // sticky FLTOP_ST_* bits
+  double offset;      // log-probability of the renormalisation point (see decode kernel)
+  int32_t pad[2];
+};
+constexpr int kStateHeaderWords = sizeof(StateHeader) / 4;
+// beam arrays stored after the header, each K words (child_filter: 2K words):
+// node, last, par, parnode, pb, pnb, first, len, child_filter
+constexpr int kStateWordsPerSlot = 10;
+inline size_t state_words(int K) { return kStateHeaderWords + (size_t)kStateWordsPerSlot * K; }
+
+struct PruneParams {
+  const float* logp;
+  int64_t stride_b, stride_t;
+  const int32_t* lengths;   // [B]
+  int32_t B, T, V;
+  float log_r;
+  int32_t* counts;          // [B*T]
+  Survivor* entries;        // [B*T*V]
+};
+
+struct DecodeParams {
+  const int32_t* lengths;   // [B] frames to consume in this call
+  const uint8_t* flags;     // [B] streaming flags or null
+  int32_t B, T, V, K, blank, L;
+  int32_t streaming;        // 0: reset at entry, no state kept.  1: state loaded / stored
+  int32_t emit_default;     // streaming with flags == null: emit results?
+  const int32_t* counts;    // [B*T] survivors per frame
+  const Survivor* entries;  // [B*T*V]
+  TrieNode* nodes;          // [B * nodes_per_utt]
+  int64_t nodes_per_utt;
+  int32_t* state;           // [B * state_words(K)] (streaming only)
+  int32_t* out_tokens;      // [B,K,L] or null
+  int32_t* out_lens;        // [B,K]
+  float* out_scores;        // [B,K]
+  int32_t* out_nhyp;        // [B]
+  int32_t* out_status;      // [B] or null
+};
+
+size_t decode_smem_bytes(int K, int V);
+int decode_block_threads(int K, int V);
+cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
+cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s);
+cudaError_t decode_prepare(int K, int V);  // one-time kernel attribute set-up
+
+}  // namespace fltop

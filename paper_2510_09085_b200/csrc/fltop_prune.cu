@@ -1,0 +1,170 @@
+// Frame-level token pruning (Algorithm 1, the conditional break; Section 3):
+// a token survives a frame iff  logp >= logp_max + log R  (float32 add and
+// compare).  Output per frame: the survivor count and the survivors as
+// {token, logp} pairs in ascending token order.
+//
+// This is the one stage that streams the emissions from HBM.  A row is read
+// exactly once with 128-bit loads, kept in registers while the row maximum is
+// reduced with warp shuffles, and compacted with ballot + popc, so the kernel
+// moves 4*V bytes in and 8*S + 4 bytes out per frame.
+#include "fltop_internal.h"
+
+namespace fltop {
+namespace {
+
+constexpr int kPruneThreads = 256;
+
+__device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
+
+__device__ __forceinline__ bool row_is_live(const PruneParams& p, int64_t row, int& b, int& t) {
+  b = (int)(row / p.T);
+  t = (int)(row - (int64_t)b * p.T);
+  int len = p.lengths[b];
+  return len <= p.T && t < len;  // a negative or oversized length reads nothing
+}
+
+// LPR lanes cooperate on one row (LPR a power of two <= 32); every lane holds
+// CH float4: tokens 4*LPR*i + 4*sub + j for i < CH, j < 4.
+template <int LPR, int CH>
+__global__ void __launch_bounds__(kPruneThreads) prune_vec_kernel(PruneParams p) {
+  constexpr int ROWS_PER_WARP = 32 / LPR;
+  const int lane = threadIdx.x & 31;
+  const int sub = lane % LPR;
+  const int grp = lane / LPR;
+  const unsigned grp_mask = (0xffffffffu >> (32 - LPR)) << (grp * LPR);
+  const unsigned lt_mask = ((1u << sub) - 1u);  // lanes of my group before me
+  const int64_t n_rows = (int64_t)p.B * p.T;
+  const int64_t warp_global = (int64_t)blockIdx.x * (kPruneThreads / 32) + (threadIdx.x >> 5);
+  const int64_t warp_stride = (int64_t)gridDim.x * (kPruneThreads / 32);
+
+  for (int64_t row0 = warp_global * ROWS_PER_WARP; row0 < n_rows;
+       row0 += warp_stride * ROWS_PER_WARP) {
+    const int64_t row = row0 + grp;
+    int b = 0, t = 0;
+    const bool live = row < n_rows && row_is_live(p, row, b, t);
+    float4 x[CH];
+    float m = neg_inf();
+    const float* src = p.logp + (int64_t)b * p.stride_b + (int64_t)t * p.stride_t;
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int tok0 = 4 * LPR * i + 4 * sub;
+      if (live && tok0 < p.V) {
+        x[i] = __ldcs(reinterpret_cast<const float4*>(src + tok0));
+      } else {
+        x[i] = make_float4(neg_inf(), neg_inf(), neg_inf(), neg_inf());
+      }
+      m = fmaxf(m, fmaxf(fmaxf(x[i].x, x[i].y), fmaxf(x[i].z, x[i].w)));
+    }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    const float thr = __fadd_rn(m, p.log_r);
+
+    Survivor* dst = p.entries + row * p.V;
+    int base = 0;
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int tok0 = 4 * LPR * i + 4 * sub;
+      const bool in = live && tok0 < p.V;
+      const float v[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
+      bool k[4];
+      unsigned bal[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        k[j] = in && v[j] >= thr;
+        bal[j] = __ballot_sync(0xffffffffu, k[j]) & grp_mask;
+      }
+      // survivors of my group held by earlier lanes in this chunk
+      const unsigned shifted_lt = lt_mask << (grp * LPR);
+      int pos = base;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) pos += __popc(bal[j] & shifted_lt);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (k[j]) {
+          dst[pos] = Survivor{tok0 + j, v[j]};
+          ++pos;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) base += __popc(bal[j]);
+    }
+    if (sub == 0 && row < n_rows) p.counts[row] = base;
+  }
+}
+
+// Any V, any alignment: one warp per row, two passes over the row (the second
+// pass is served by L1/L2).
+__global__ void __launch_bounds__(kPruneThreads) prune_scalar_kernel(PruneParams p) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n_rows = (int64_t)p.B * p.T;
+  const int64_t warp_global = (int64_t)blockIdx.x * (kPruneThreads / 32) + (threadIdx.x >> 5);
+  const int64_t warp_stride = (int64_t)gridDim.x * (kPruneThreads / 32);
+  for (int64_t row = warp_global; row < n_rows; row += warp_stride) {
+    int b, t;
+    const bool live = row_is_live(p, row, b, t);
+    if (!live) {
+      if (lane == 0) p.counts[row] = 0;
+      continue;
+    }
+    const float* src = p.logp + (int64_t)b * p.stride_b + (int64_t)t * p.stride_t;
+    float m = neg_inf();
+    for (int c = lane; c < p.V; c += 32) m = fmaxf(m, src[c]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    const float thr = __fadd_rn(m, p.log_r);
+    Survivor* dst = p.entries + row * p.V;
+    int base = 0;
+    for (int c0 = 0; c0 < p.V; c0 += 32) {
+      const int c = c0 + lane;
+      const float v = c < p.V ? src[c] : neg_inf();
+      const bool k = c < p.V && v >= thr;
+      const unsigned bal = __ballot_sync(0xffffffffu, k);
+      if (k) dst[base + __popc(bal & ((1u << lane) - 1u))] = Survivor{c, v};
+      base += __popc(bal);
+    }
+    if (lane == 0) p.counts[row] = base;
+  }
+}
+
+template <int LPR, int CH>
+cudaError_t launch_vec(const PruneParams& p, cudaStream_t s, int sms) {
+  const int64_t n_rows = (int64_t)p.B * p.T;
+  const int rows_per_block = (kPruneThreads / 32) * (32 / LPR);
+  int64_t blocks = (n_rows + rows_per_block - 1) / rows_per_block;
+  const int64_t cap = (int64_t)sms * 8;  // 8 resident blocks of 256 threads per SM
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  prune_vec_kernel<LPR, CH><<<(unsigned)blocks, kPruneThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_prune(const PruneParams& p, cudaStream_t s) {
+  if ((int64_t)p.B * p.T == 0) return cudaSuccess;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const bool aligned = (p.V % 4 == 0) && (p.stride_b % 4 == 0) && (p.stride_t % 4 == 0) &&
+                       ((reinterpret_cast<uintptr_t>(p.logp) & 15u) == 0);
+  if (aligned) {
+    const int quads = p.V / 4;
+    if (quads <= 1) return launch_vec<1, 1>(p, s, sms);
+    if (quads <= 2) return launch_vec<2, 1>(p, s, sms);
+    if (quads <= 4) return launch_vec<4, 1>(p, s, sms);
+    if (quads <= 8) return launch_vec<8, 1>(p, s, sms);
+    if (quads <= 16) return launch_vec<16, 1>(p, s, sms);
+    if (quads <= 32) return launch_vec<32, 1>(p, s, sms);
+    if (quads <= 64) return launch_vec<32, 2>(p, s, sms);
+    if (quads <= 128) return launch_vec<32, 4>(p, s, sms);
+    if (quads <= 256) return launch_vec<32, 8>(p, s, sms);
+    if (quads <= 512) return launch_vec<32, 16>(p, s, sms);
+  }
+  const int64_t n_rows = (int64_t)p.B * p.T;
+  int64_t blocks = (n_rows + (kPruneThreads / 32) - 1) / (kPruneThreads / 32);
+  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+  prune_scalar_kernel<<<(unsigned)blocks, kPruneThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace fltop
