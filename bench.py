@@ -1,0 +1,330 @@
+"""Benchmark of the frame-pruned CTC prefix beam search library.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole hot path (prune, extend, merge, select, trie
+append, readback) over one synthetic wav2vec2-shaped batch: B=64 utterances,
+T uniform in [250, 1750], V=32, beam 50, R=1e-3.  The same input is also
+decoded at R=0 (no pruning) and both are reported.  The emissions are 14 MB,
+far below L2, so a buffer larger than L2 is written between timed steps.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "frames/sec decoded (batch 64, beam 50, r=1e-3 vs r=0); % HBM roofline"
+UNIT = "frames/s"
+BATCH, BEAM, R_PRUNED = 64, 50, 1e-3
+L2_FLUSH_BYTES = 256 << 20
+NODE_BYTES, SURVIVOR_BYTES = 32, 8
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-i", str(gpu_index), "-lms", "50"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def _workload(rank: int):
+    from paper_2510_09085_b200 import workloads
+    return workloads.workload_wav2vec2(seed=1 + 1000 * rank, batch=BATCH, beam_width=BEAM)
+
+
+def _oracle_frames_per_s(wl, r, utterances):
+    """The CPU oracle, as it stands, single thread, on a subset of the utterances."""
+    import oracle
+    em, ln = wl.emissions[utterances], wl.lengths[utterances]
+    t0 = time.perf_counter()
+    oracle.decode(em, ln, wl.blank_id, wl.beam_width, r)
+    dt = time.perf_counter() - t0
+    return float(ln.sum()) / dt, dt
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: each step decodes a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = _workload(0)
+    order = np.argsort(wl.lengths)
+    sample = [int(i) for i in order[::8]]          # 8 utterances spread over the length range
+    for _ in range(args.warmup):
+        _oracle_frames_per_s(wl, R_PRUNED, sample[:1])
+    frames, total = 0.0, 0.0
+    for _ in range(args.steps):
+        fps, dt = _oracle_frames_per_s(wl, R_PRUNED, sample)
+        frames += fps * dt
+        total += dt
+    value = frames / total
+    desc = f"{len(sample)} of {BATCH} utterances per step, r=1e-3, K={BEAM}"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": BATCH, "beam": BEAM, "r": R_PRUNED,
+                   "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+    from paper_2510_09085_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+    if not torch.cuda.is_available():
+        raise SystemExit("no CUDA device: this benchmark has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    wl = _workload(rank)
+    B, T, V = wl.emissions.shape
+    n_frames = int(wl.lengths.sum())
+    host_em = torch.from_numpy(wl.emissions).pin_memory()
+    host_ln = torch.from_numpy(wl.lengths).pin_memory()
+    dev_em = host_em.cuda()
+    dev_ln = host_ln.cuda()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+
+    def make(r):
+        d = binding.Decoder(V, wl.blank_id, BEAM, r, B, T, device=local_rank)
+        d.set_profiling(True)
+        return d
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(dec, steps, warmup, e2e=False):
+        """Per-step device times (ms) of `steps` decodes; warm-up steps are not timed."""
+        out_host = None
+        if e2e:
+            out_host = [torch.empty_like(t, device="cpu").pin_memory()
+                        for t in (dec.tokens, dec.lens, dec.scores, dec.nhyp)]
+        step_ms, prune_ms, decode_ms = [], [], []
+        launches0 = 0
+        with torch.cuda.stream(stream):
+            for i in range(warmup + steps):
+                if i == warmup:
+                    barrier()
+                    launches0 = dec.launch_count
+                flush.fill_(i & 0xff)                      # evict the inputs from L2
+                t0, t1 = torch.cuda.Event(True), torch.cuda.Event(True)
+                t0.record(stream)
+                if e2e:
+                    dev_em.copy_(host_em, non_blocking=True)
+                    dev_ln.copy_(host_ln, non_blocking=True)
+                dec.decode(dev_em, dev_ln, stream=stream)
+                if e2e:
+                    for h, d in zip(out_host, (dec.tokens, dec.lens, dec.scores, dec.nhyp)):
+                        h.copy_(d, non_blocking=True)
+                t1.record(stream)
+                t1.synchronize()
+                if i >= warmup:
+                    step_ms.append(t0.elapsed_time(t1))
+                    pk, dk = dec.last_kernel_ms()
+                    prune_ms.append(pk)
+                    decode_ms.append(dk)
+            barrier()
+        return step_ms, prune_ms, decode_ms, dec.launch_count - launches0
+
+    def reduce_max(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def reduce_sum(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    dec_p, dec_0 = make(R_PRUNED), make(0.0)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms_p, prune_p, decode_p, launches = timed(dec_p, args.steps, args.warmup)
+    clocks = sampler.stop() if sampler else None
+    ms_0, prune_0, decode_0, _ = timed(dec_0, args.steps, args.warmup)
+    ms_e, _, _, _ = timed(dec_p, args.steps, args.warmup, e2e=True)
+
+    total_frames = reduce_sum(float(n_frames))
+    t_p = reduce_max(sum(ms_p)) / args.steps
+    t_0 = reduce_max(sum(ms_0)) / args.steps
+    t_e = reduce_max(sum(ms_e)) / args.steps
+    stats_p = dec_p.last_call_stats()
+    stats_0 = dec_0.last_call_stats()
+    assert int((dec_p.status != 0).sum()) == 0 and int((dec_0.status != 0).sum()) == 0
+
+    def kernel_bytes(dec, st):
+        """Algorithmic HBM bytes of one launch of each kernel (inputs of this rank)."""
+        n_hyp = int(dec.nhyp.sum())
+        out_bytes = 4 * int(dec.lens.sum()) + 8 * n_hyp + 8 * B
+        prune = st["frames"] * (4 * V + 4) + st["survivors"] * SURVIVOR_BYTES
+        decode = (st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES
+                  + st["trie_nodes_created"] * (NODE_BYTES + 12) + out_bytes)
+        return prune, decode
+
+    peak, peak_kind = _peaks()
+    pb, db = kernel_bytes(dec_p, stats_p)
+    pb0, db0 = kernel_bytes(dec_0, stats_0)
+    dk_ms = statistics.mean(decode_p)
+    achieved = db / (dk_ms * 1e-3) / 1e9
+    h2d = host_em.numel() * 4 + host_ln.numel() * 4
+    d2h = sum(t.numel() * t.element_size() for t in (dec_p.tokens, dec_p.lens, dec_p.scores,
+                                                     dec_p.nhyp))
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        fps, dt = _oracle_frames_per_s(wl, R_PRUNED, list(range(B)))
+        order = np.argsort(wl.lengths)
+        fps0, dt0 = _oracle_frames_per_s(wl, 0.0, [int(i) for i in order[::8]])
+        cpu = {"value": fps, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"all {B} utterances of the workload at r=1e-3 ({dt:.1f} s); "
+                         f"r=0 on 8 utterances: {fps0:.0f} frames/s ({dt0:.1f} s)",
+               "value_r0": fps0, "host_cores_available": len(os.sched_getaffinity(0))}
+
+    line = {
+        "metric": METRIC, "value": total_frames / (t_p * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_p,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "batch_per_gpu": B, "beam": BEAM, "r": R_PRUNED,
+                   "vocab": V, "frames_per_step_per_gpu": n_frames, "max_frames": int(T),
+                   "l2": f"flushed: {L2_FLUSH_BYTES >> 20} MiB written between timed steps",
+                   "sharding": "one independent batch per GPU, no collective"},
+        "e2e": {"value": total_frames / (t_e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": t_e},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "peak_source": f"{peak_kind} copy bandwidth",
+                     "bytes_per_launch": db, "ms_per_launch": dk_ms,
+                     "note": "latency-bound serial frame chain: max_frames dependent steps"},
+        "cpu_baseline": cpu,
+        "detail": {
+            "r0": {"value": total_frames / (t_0 * 1e-3), "ms_per_step": t_0,
+                   "decode_kernel_ms": statistics.mean(decode_0),
+                   "prune_kernel_ms": statistics.mean(prune_0),
+                   "mean_survivors": stats_0["survivors"] / max(1, stats_0["frames"]),
+                   "mean_live_hypotheses": stats_0["live_hypotheses_sum"] / max(1, stats_0["frames"]),
+                   "hbm_frac_step": (pb0 + db0) / (t_0 * 1e-3) / 1e9 / peak},
+            "pruned_over_r0_speedup": t_0 / t_p,
+            "utterances_per_s": world * B / (t_p * 1e-3),
+            "prune_kernel_ms": statistics.mean(prune_p),
+            "decode_kernel_ms": dk_ms,
+            "ns_per_frame_step": 1e6 * dk_ms / int(wl.lengths.max()),
+            "mean_survivors": stats_p["survivors"] / max(1, stats_p["frames"]),
+            "mean_live_hypotheses": stats_p["live_hypotheses_sum"] / max(1, stats_p["frames"]),
+            "trie_nodes_created": stats_p["trie_nodes_created"],
+            "hbm_frac_step": (pb + db) / (t_p * 1e-3) / 1e9 / peak,
+            "prune_kernel_gbs": pb / (statistics.mean(prune_p) * 1e-3) / 1e9,
+            "beam_state_bytes": dec_p.beam_state_bytes,
+            "step_ms_min": min(ms_p), "step_ms_median": statistics.median(ms_p),
+        },
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -138,6 +138,10 @@ int fltop_last_cuda_error(const fltop_handle* h);
 size_t fltop_beam_state_bytes(const fltop_handle* h);
 /* Kernels launched by this handle since creation. */
 int64_t fltop_launch_count(const fltop_handle* h);
+/* Totals of the most recent decode / stream_step call (synchronises its stream):
+ * out[0] frames decoded, out[1] survivors over those frames, out[2] prefix-trie nodes
+ * created, out[3] beam entries summed over frames (mean live hypotheses = out[3]/out[0]). */
+int fltop_last_call_stats(fltop_handle* h, int64_t* out);
 /* With profiling enabled every call brackets its kernels with CUDA events on the caller's
  * stream.  fltop_last_kernel_ms synchronises on those events and returns the device time
  * of the most recent call's {prune, decode} kernels in out_ms[0..1] (milliseconds). */

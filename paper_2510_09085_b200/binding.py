@@ -22,7 +22,7 @@ FLTOP_ST_BAD_LENGTH, FLTOP_ST_ARENA_FULL, FLTOP_ST_TRUNCATED, FLTOP_ST_EMPTY_BEA
 
 EXPORTS = ("fltop_workspace_size", "fltop_create", "fltop_decode", "fltop_stream_step",
            "fltop_destroy", "fltop_prune", "fltop_status_string", "fltop_last_cuda_error",
-           "fltop_beam_state_bytes", "fltop_launch_count", "fltop_set_profiling",
+           "fltop_beam_state_bytes", "fltop_launch_count", "fltop_last_call_stats", "fltop_set_profiling",
            "fltop_last_kernel_ms")
 
 
@@ -73,6 +73,8 @@ def lib():
         L.fltop_beam_state_bytes.argtypes = [vp]
         L.fltop_launch_count.restype = C.c_int64
         L.fltop_launch_count.argtypes = [vp]
+        L.fltop_last_call_stats.restype = C.c_int
+        L.fltop_last_call_stats.argtypes = [vp, C.POINTER(C.c_int64)]
         L.fltop_set_profiling.restype = C.c_int
         L.fltop_set_profiling.argtypes = [vp, C.c_int]
         L.fltop_last_kernel_ms.restype = C.c_int
@@ -214,6 +216,14 @@ class Decoder:
         if code != FLTOP_OK:
             raise FltopError(code, "fltop_last_kernel_ms")
         return float(ms[0]), float(ms[1])
+
+    def last_call_stats(self) -> dict:
+        out = (C.c_int64 * 4)()
+        code = lib().fltop_last_call_stats(self.h, out)
+        if code != FLTOP_OK:
+            raise FltopError(code, "fltop_last_call_stats")
+        return {"frames": out[0], "survivors": out[1], "trie_nodes_created": out[2],
+                "live_hypotheses_sum": out[3]}
 
     @property
     def beam_state_bytes(self) -> int:

@@ -20,6 +20,9 @@ struct fltop_handle {
   Survivor* entries;
   TrieNode* nodes;
   int32_t* state;
+  int32_t* stats;
+  int32_t last_B, last_T;
+  cudaStream_t last_stream;
   int64_t frame_cap;      // frames per utterance the survivor buffers hold
   int64_t nodes_per_utt;
   size_t beam_state_bytes;
@@ -56,7 +59,7 @@ bool config_ok(const fltop_config* c) {
 }
 
 struct Layout {
-  size_t counts, entries, nodes, state, total, beam_state;
+  size_t counts, entries, nodes, state, stats, total, beam_state;
   int64_t frame_cap, nodes_per_utt;
 };
 
@@ -71,8 +74,9 @@ Layout layout_of(const fltop_config& c) {
   l.nodes = off; off += up((size_t)c.max_batch * (size_t)l.nodes_per_utt * sizeof(TrieNode));
   l.state = off;
   if (c.max_chunk_frames > 0) off += up((size_t)c.max_batch * state_words(c.beam_width) * 4);
-  l.total = off;
   l.beam_state = off;  // survivor lists + trie arenas + stream states
+  l.stats = off; off += up((size_t)c.max_batch * 4 * sizeof(int32_t));
+  l.total = off;  // survivor lists + trie arenas + stream states
   return l;
 }
 
@@ -122,6 +126,8 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
   dp.out_status = d_status;
+  dp.stats = h->stats;
+  h->last_B = B; h->last_T = T; h->last_stream = s;
 
   if (h->profiling) cudaEventRecord(h->ev[0], s);
   if (T > 0) {
@@ -190,6 +196,8 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   h->entries = reinterpret_cast<Survivor*>(h->ws + l.entries);
   h->nodes = reinterpret_cast<TrieNode*>(h->ws + l.nodes);
   h->state = cfg->max_chunk_frames > 0 ? reinterpret_cast<int32_t*>(h->ws + l.state) : nullptr;
+  h->stats = reinterpret_cast<int32_t*>(h->ws + l.stats);
+  h->last_B = 0; h->last_T = 0; h->last_stream = nullptr;
   h->frame_cap = l.frame_cap;
   h->nodes_per_utt = l.nodes_per_utt;
   h->beam_state_bytes = l.beam_state;
@@ -290,6 +298,33 @@ const char* fltop_status_string(int code) {
 int fltop_last_cuda_error(const fltop_handle* h) { return h ? h->last_cuda : 0; }
 size_t fltop_beam_state_bytes(const fltop_handle* h) { return h ? h->beam_state_bytes : 0; }
 int64_t fltop_launch_count(const fltop_handle* h) { return h ? h->launches : 0; }
+
+int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
+  if (!h || !out) return FLTOP_ERR_INVALID_ARG;
+  out[0] = out[1] = out[2] = out[3] = 0;
+  if (h->last_B == 0) return FLTOP_OK;
+  DeviceGuard g;
+  cudaError_t e = g.enter(h->cfg.device);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(h->last_stream);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  const size_t B = (size_t)h->last_B, n_frames = B * (size_t)h->last_T;
+  int32_t* host = new (std::nothrow) int32_t[4 * B + n_frames];
+  if (!host) return FLTOP_ERR_OOM;
+  e = cudaMemcpy(host, h->stats, 4 * B * sizeof(int32_t), cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && n_frames)
+    e = cudaMemcpy(host + 4 * B, h->counts, n_frames * sizeof(int32_t), cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) {
+    for (size_t b = 0; b < B; ++b) {
+      out[0] += host[4 * b];
+      out[2] += host[4 * b + 1];
+      out[3] += host[4 * b + 2];
+    }
+    for (size_t i = 0; i < n_frames; ++i) out[1] += host[4 * B + i];
+  }
+  delete[] host;
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  return FLTOP_OK;
+}
 
 int fltop_set_profiling(fltop_handle* h, int enable) {
   if (!h) return FLTOP_ERR_INVALID_ARG;

@@ -94,7 +94,7 @@ struct Smem {
 };
 enum {
   SC_NBEAM_NEXT = 0, SC_MAXKEY, SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_REVIVED,
-  SC_STATUS, SC_BLANK_J, SC_COUNT
+  SC_STATUS, SC_BLANK_J, SC_CREATED, SC_COUNT
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -258,7 +258,9 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
     S.scal[SC_BLANK_J] = -1;
     S.scal[SC_REVIVED] = 0;
     S.scal[SC_STATUS] = 0;
+    S.scal[SC_CREATED] = 0;
   }
+  int created = 0, live_sum = 0;
   int cur = 0, nb, n_nodes, frames_seen;
   double offset;
   if (do_reset) {
@@ -539,6 +541,7 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
           n.depth = N.len[s]; n.pad = 0; n.child_filter = 0ull;
           nodes[id] = n;
           N.node[s] = id;
+          ++created;
         } else {
           N.node[s] = 0;
           S.scal[SC_STATUS] = 2;  // FLTOP_ST_ARENA_FULL
@@ -576,6 +579,7 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
     if (!maxkey) status |= 8;  // FLTOP_ST_EMPTY_BEAM
     offset += (double)best;
     n_nodes += nbn;
+    live_sum += nbn;
     nb = nbn;
     cur ^= 1;
     cnt0 = cnt1;
@@ -585,6 +589,14 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
   }
   frames_seen += len;
   status |= S.scal[SC_STATUS];
+  if (p.stats) {
+    if (created) atomicAdd(&S.scal[SC_CREATED], created);
+    __syncthreads();
+    if (tid == 0) {
+      int32_t* o = p.stats + 4 * (int64_t)b;
+      o[0] = len; o[1] = S.scal[SC_CREATED]; o[2] = live_sum; o[3] = n_nodes;
+    }
+  }
 
   Beam& F = S.beam[cur];
 

@@ -67,6 +67,7 @@ struct DecodeParams {
   float* out_scores;        // [B,K]
   int32_t* out_nhyp;        // [B]
   int32_t* out_status;      // [B] or null
+  int32_t* stats;           // [B,4] frames, trie nodes created, sum of beam sizes, node ids used; or null
 };
 
 size_t decode_smem_bytes(int K, int V);
