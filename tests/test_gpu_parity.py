@@ -205,3 +205,40 @@ def test_host_side_argument_errors():
     assert bd.fltop_decode(h2, x, 3200, 32, ln, 4, 100, tok, le, sc, nh) == bd.FLTOP_OK
     torch.cuda.synchronize()
     assert bd.fltop_destroy(h2) == bd.FLTOP_OK
+
+
+# ------------------------------------------------------------------ crowded cut / ties
+def test_many_near_equal_scores_take_the_exact_select_path():
+    # nearly flat rows: the candidates of a frame fall into very few score-histogram
+    # bins, so the cut bin holds far more members than the pairwise ranking handles
+    rng = np.random.default_rng(5)
+    B, T, V = 3, 14, 16
+    x = rng.standard_normal((B, T, V)) * 0.02
+    em = (x - np.log(np.exp(x).sum(-1, keepdims=True))).astype(np.float32)
+    ln = np.array([T, T - 3, 5], dtype=np.int32)
+    for K, r in [(8, 0.0), (20, 0.5), (100, 0.0)]:
+        d = gpu_decode(em, ln, 0, K, r)
+        res = oracle.decode(em, ln, 0, K, r)
+        for b in range(B):
+            check_hyps(d.hyps(b), res.hyps(b), K, max_unmatched_frac=0.3,
+                       where=f"flat utt {b} K={K}")
+        d.close()
+
+
+def test_exact_ties_keep_a_valid_beam():
+    # constant rows: every extension of a prefix ties exactly.  Which of the tied
+    # candidates survive is not unique; every kept hypothesis must carry its exact
+    # score and no dropped hypothesis may beat a kept one.
+    T, V, K = 5, 4, 6
+    em = np.full((1, T, V), np.log(1.0 / V), dtype=np.float32)
+    ln = np.array([T], dtype=np.int32)
+    full = dict(oracle.decode(em, ln, 0, 100000, 0.0).hyps(0))      # every labelling, exact
+    d = gpu_decode(em, ln, 0, K, 0.0)
+    ref = oracle.decode(em, ln, 0, K, 0.0).hyps(0)
+    got = d.hyps(0)
+    assert len(got) == K and len(set(s for s, _ in got)) == K
+    # finite-beam scores are lower bounds of the exact ones and the score lists agree
+    for seq, sc in got:
+        assert sc <= full[seq] + TOL
+    np.testing.assert_allclose(sorted(s for _, s in got), sorted(s for _, s in ref), atol=TOL)
+    d.close()
