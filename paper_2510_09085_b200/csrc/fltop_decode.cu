@@ -363,7 +363,7 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
       bi(0, F_NODE)[i] = a[i]; bi(0, F_LAST)[i] = a[K + i]; bi(0, F_PAR)[i] = a[2 * K + i];
       bi(0, F_PARNODE)[i] = a[3 * K + i];
       const float pb = __int_as_float(a[4 * K + i]), pnb = __int_as_float(a[5 * K + i]);
-      bf(0, F_PB)[i] = pb; bf(0, F_PNB)[i] = pnb; bf(0, F_TOT)[i] = lse2(pb, pnb);
+      bf(0, F_PB)[i] = pb; bf(0, F_PNB)[i] = pnb; bf(0, F_TOT)[i] = __int_as_float(a[10 * K + i]);
       bi(0, F_FIRST)[i] = a[6 * K + i]; bi(0, F_LEN)[i] = a[7 * K + i];
       filt(0)[i] = reinterpret_cast<const unsigned long long*>(a + 8 * K)[i];
     }
@@ -776,6 +776,7 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
       a[4 * K + i] = bi(cur, F_PB)[i]; a[5 * K + i] = bi(cur, F_PNB)[i];
       a[6 * K + i] = bi(cur, F_FIRST)[i]; a[7 * K + i] = bi(cur, F_LEN)[i];
       reinterpret_cast<unsigned long long*>(a + 8 * K)[i] = filt(cur)[i];
+      a[10 * K + i] = bi(cur, F_TOT)[i];
     }
     if (tid == 0) {
       StateHeader* hd = reinterpret_cast<StateHeader*>(st);

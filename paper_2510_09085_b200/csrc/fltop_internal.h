@@ -37,8 +37,8 @@ struct StateHeader {
 };
 constexpr int kStateHeaderWords = sizeof(StateHeader) / 4;
 // beam arrays stored after the header, each K words (child_filter: 2K words):
-// node, last, par, parnode, pb, pnb, first, len, child_filter
-constexpr int kStateWordsPerSlot = 10;
+// node, last, par, parnode, pb, pnb, first, len, child_filter (2 words), tot
+constexpr int kStateWordsPerSlot = 11;
 inline size_t state_words(int K) { return kStateHeaderWords + (size_t)kStateWordsPerSlot * K; }
 
 struct PruneParams {
