@@ -130,6 +130,38 @@ int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t 
                 const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_counts,
                 void* d_entries, void* cuda_stream);
 
+/* Batch decode without any allocation.  The paper has no counterpart to this call: it exists
+ * for callers that cannot call cudaMalloc where they decode - a real-time audio thread that
+ * must not block in the driver's allocator, a plug-in living inside another framework's
+ * memory pool with a fixed budget, a process that has already given all device memory to a
+ * caching allocator.  It computes exactly what fltop_create + fltop_decode + fltop_destroy
+ * compute, but its scratch (survivor lists, prefix-trie arena) is a fixed array inside the
+ * library image, FLTOP_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the
+ * process exits.  Consequently:
+ *   - the problem must fit: vocab_size <= FLTOP_STATIC_MAX_VOCAB, B*T <=
+ *     FLTOP_STATIC_MAX_FRAMES, B*(beam_width*T + 1) <= FLTOP_STATIC_MAX_NODES; anything
+ *     larger returns FLTOP_ERR_CAPACITY and launches nothing;
+ *   - it runs on the CURRENT device.  The first call on each device looks up the array's
+ *     device address (cudaGetSymbolAddress) before launching; make that first call outside
+ *     any stream capture;
+ *   - all calls share the one array.  It needs no clearing between calls (every word a
+ *     call reads it has written first), but two calls whose kernels overlap on the GPU -
+ *     different streams, or different host threads - race on it.  Serialise them.
+ *   - it calls no cudaMalloc / cudaFree and no allocating library routine; inputs and
+ *     outputs are the caller's device buffers, with the meaning they have in fltop_decode
+ *     (d_tokens is [B, beam_width, max_out_len]). */
+#define FLTOP_STATIC_MAX_VOCAB 64
+#define FLTOP_STATIC_MAX_FRAMES 4096
+#define FLTOP_STATIC_MAX_NODES 131072
+#define FLTOP_STATIC_SCRATCH_BYTES \
+  (FLTOP_STATIC_MAX_FRAMES * 4 + FLTOP_STATIC_MAX_FRAMES * FLTOP_STATIC_MAX_VOCAB * 8 + \
+   FLTOP_STATIC_MAX_NODES * 32)
+int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t beam_width,
+                        float threshold_r, const float* d_logp, int64_t stride_b,
+                        int64_t stride_t, const int32_t* d_lengths, int32_t B, int32_t T,
+                        int32_t max_out_len, int32_t* d_tokens, int32_t* d_lens, float* d_scores,
+                        int32_t* d_nhyp, int32_t* d_status, void* cuda_stream);
+
 /* Optional helpers. */
 const char* fltop_status_string(int code);
 /* Last cudaError_t seen by this handle (0 if none). */

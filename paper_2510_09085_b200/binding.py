@@ -23,7 +23,7 @@ FLTOP_ST_BAD_LENGTH, FLTOP_ST_ARENA_FULL, FLTOP_ST_TRUNCATED, FLTOP_ST_EMPTY_BEA
 EXPORTS = ("fltop_workspace_size", "fltop_create", "fltop_decode", "fltop_stream_step",
            "fltop_destroy", "fltop_prune", "fltop_status_string", "fltop_last_cuda_error",
            "fltop_beam_state_bytes", "fltop_launch_count", "fltop_last_call_stats", "fltop_set_profiling",
-           "fltop_last_kernel_ms")
+           "fltop_last_kernel_ms", "fltop_decode_static")
 
 
 class fltop_config(C.Structure):
@@ -79,6 +79,9 @@ def lib():
         L.fltop_set_profiling.argtypes = [vp, C.c_int]
         L.fltop_last_kernel_ms.restype = C.c_int
         L.fltop_last_kernel_ms.argtypes = [vp, C.POINTER(C.c_float)]
+        L.fltop_decode_static.restype = C.c_int
+        L.fltop_decode_static.argtypes = [i32, i32, i32, C.c_float, vp, i64, i64, vp, i32, i32,
+                                          i32, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -136,6 +139,16 @@ def fltop_stream_step(h, chunk, chunk_lens, flags, S, Cf, tokens, lens, scores, 
 def fltop_prune(h, logp, stride_b, stride_t, lengths, B, T, counts, entries, stream=None) -> int:
     return lib().fltop_prune(h, _p(logp), stride_b, stride_t, _p(lengths), B, T, _p(counts),
                              _p(entries), _stream_ptr(stream))
+
+
+def fltop_decode_static(vocab_size, blank_id, beam_width, threshold_r, logp, stride_b, stride_t,
+                        lengths, B, T, max_out_len, tokens, lens, scores, nhyp, status=None,
+                        stream=None) -> int:
+    """Allocation-free batch decode on the current device (fixed scratch inside the library)."""
+    return lib().fltop_decode_static(vocab_size, blank_id, beam_width, threshold_r, _p(logp),
+                                     stride_b, stride_t, _p(lengths), B, T, max_out_len,
+                                     _p(tokens), _p(lens), _p(scores), _p(nhyp), _p(status),
+                                     _stream_ptr(stream))
 
 
 def fltop_destroy(h) -> int:
