@@ -30,7 +30,7 @@ METRIC = "frames/sec decoded (batch 64, beam 50, r=1e-3 vs r=0); % HBM roofline"
 UNIT = "frames/s"
 BATCH, BEAM, R_PRUNED = 64, 50, 1e-3
 L2_FLUSH_BYTES = 256 << 20
-NODE_BYTES, SURVIVOR_BYTES = 32, 8
+NODE_BYTES, SURVIVOR_BYTES = 8, 8
 
 
 def _peaks():
@@ -241,8 +241,10 @@ def run_ours(args):
         n_hyp = int(dec.nhyp.sum())
         out_bytes = 4 * int(dec.lens.sum()) + 8 * n_hyp + 8 * B
         prune = st["frames"] * (4 * V + 4) + st["survivors"] * SURVIVOR_BYTES
-        decode = (st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES
-                  + st["trie_nodes_created"] * (NODE_BYTES + 12) + out_bytes)
+        # survivor lists read back, one block of 8-byte trie records per frame (one record
+        # per beam slot, rounded up to an even count), the hypotheses written at the end
+        trie = NODE_BYTES * (st["live_hypotheses_sum"] + st["frames"])
+        decode = st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES + trie + out_bytes
         return prune, decode
 
     peak, peak_kind = _peaks()

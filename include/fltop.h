@@ -155,7 +155,7 @@ int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t 
 #define FLTOP_STATIC_MAX_NODES 131072
 #define FLTOP_STATIC_SCRATCH_BYTES \
   (FLTOP_STATIC_MAX_FRAMES * 4 + FLTOP_STATIC_MAX_FRAMES * FLTOP_STATIC_MAX_VOCAB * 8 + \
-   FLTOP_STATIC_MAX_NODES * 32)
+   FLTOP_STATIC_MAX_NODES * 8)
 int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t beam_width,
                         float threshold_r, const float* d_logp, int64_t stride_b,
                         int64_t stride_t, const int32_t* d_lengths, int32_t B, int32_t T,
@@ -178,6 +178,9 @@ int fltop_last_call_stats(fltop_handle* h, int64_t* out);
  * stream.  fltop_last_kernel_ms synchronises on those events and returns the device time
  * of the most recent call's {prune, decode} kernels in out_ms[0..1] (milliseconds). */
 int fltop_set_profiling(fltop_handle* h, int enable);
+/* Threads per utterance block of the decode kernel (a multiple of 32, at most 1024; 0 = let
+ * the library choose from K, V and R).  A tuning knob: results do not depend on it. */
+int fltop_set_block_threads(fltop_handle* h, int32_t threads);
 int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
 
 #ifdef __cplusplus

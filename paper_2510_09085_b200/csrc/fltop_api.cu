@@ -28,6 +28,7 @@ struct fltop_handle {
   size_t beam_state_bytes;
   int last_cuda;
   int64_t launches;
+  int32_t block_threads;  // 0 = chosen by the library
   bool profiling;
   bool prof_valid;
   cudaEvent_t ev[3];
@@ -51,7 +52,7 @@ bool config_ok(const fltop_config* c) {
   if (c->top_n != 0) return false;
   if (c->beam_threshold > 0.f || c->beam_threshold != c->beam_threshold) return false;
   if (c->device < 0) return false;
-  if ((int64_t)c->beam_width * c->max_frames + 1 > (int64_t)std::numeric_limits<int32_t>::max())
+  if ((int64_t)(c->beam_width + 1) * c->max_frames + 2 > (int64_t)std::numeric_limits<int32_t>::max())
     return false;
   if (decode_smem_bytes(c->beam_width, c->vocab_size) > kMaxSmem) return false;
   if (c->workspace && (reinterpret_cast<uintptr_t>(c->workspace) % kAlign) != 0) return false;
@@ -66,7 +67,8 @@ struct Layout {
 Layout layout_of(const fltop_config& c) {
   Layout l;
   l.frame_cap = c.max_chunk_frames > 0 ? c.max_chunk_frames : c.max_frames;
-  l.nodes_per_utt = (int64_t)c.beam_width * c.max_frames + 1;
+  // a frame takes an even-sized block of at most beam_width node ids; ids 0 and 1 are fixed
+  l.nodes_per_utt = (int64_t)((c.beam_width + 1) & ~1) * c.max_frames + 2;
   const size_t frames = (size_t)c.max_batch * (size_t)l.frame_cap;
   size_t off = 0;
   l.counts = off; off += up(frames * sizeof(int32_t));
@@ -122,6 +124,7 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.lengths = d_lengths; dp.flags = d_flags; dp.B = B; dp.T = T; dp.V = h->cfg.vocab_size;
   dp.K = h->cfg.beam_width; dp.blank = h->cfg.blank_id; dp.L = h->cfg.max_out_len;
   dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
+  dp.block_threads = h->block_threads; dp.pruning = h->cfg.threshold_r > 0.f ? 1 : 0;
   dp.counts = h->counts; dp.entries = h->entries; dp.nodes = h->nodes;
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
@@ -176,6 +179,7 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   h->log_r = cfg->threshold_r > 0.f ? (float)std::log((double)cfg->threshold_r)
                                     : -std::numeric_limits<float>::infinity();
   h->last_cuda = 0; h->launches = 0; h->profiling = false; h->prof_valid = false;
+  h->block_threads = 0;
   h->ev[0] = h->ev[1] = h->ev[2] = nullptr;
   if (cfg->workspace) {
     h->ws = static_cast<unsigned char*>(cfg->workspace);
@@ -323,6 +327,12 @@ int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
   }
   delete[] host;
   if (e != cudaSuccess) return cuda_fail(h, e);
+  return FLTOP_OK;
+}
+
+int fltop_set_block_threads(fltop_handle* h, int32_t threads) {
+  if (!h || threads < 0 || threads > 1024 || threads % 32 != 0) return FLTOP_ERR_INVALID_ARG;
+  h->block_threads = threads;
   return FLTOP_OK;
 }
 

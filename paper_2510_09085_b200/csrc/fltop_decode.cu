@@ -5,49 +5,91 @@
 //
 // One thread block decodes one utterance and walks its frames serially; the
 // beam lives in shared memory for the whole utterance.  The frame loop is a
-// chain of dependent steps, so the design minimises block barriers per frame
-// (five on the common path) rather than bytes moved:
-//   P1  every beam entry q gets its "stay" candidate (pb' = tot + lp[blank],
-//       pnb' = pnb + lp[last(q)], plus - the prefix merge - the mass of its
-//       parent extended by last(q) when the parent is in the beam); every
-//       (beam entry, non-blank survivor) pair gets an extension candidate
-//       unless that prefix is already in the beam.  Each candidate adds one
-//       to a 512-bin histogram of its score (1/8 nat per bin).
-//   P2  warp 0 scans the histogram: the bin holding the K-th best score is
-//       the cut; bins above it become slot counters.  Meanwhile the other
-//       warps publish last frame's trie changes and stage the next frame's
-//       log-probabilities.
-//   P3  candidates above the cut take their beam slot with one shared-memory
-//       atomic and are written to the next beam; candidates inside the cut
-//       bin are ranked exactly among themselves (a handful).
-//   P5  selected extensions get their trie node by lookup-or-create, so that
-//       one node id always means one token sequence; parent slots and the
-//       in-beam child bits of the next frame are set.
+// chain of dependent steps and nothing in it is bandwidth-bound: what bounds a
+// frame is the longest chain of dependent instructions any one warp runs
+// between two barriers.  The warps of a block therefore have roles:
+//
+//   stay warps   one lane per beam entry q: the "stay" candidate
+//                (pb' = tot + lp[blank], pnb' = pnb + lp[last(q)]) and the
+//                prefix merge.
+//   ext warps    the (beam entry, non-blank survivor) extension candidates,
+//                dealt out so that candidate e = q * S + j goes to ext lane
+//                e mod NX; the extensions that end up selected come from the
+//                few best entries, i.e. from consecutive e, and so land on
+//                different lanes.
+//   chore warp   everything a frame needs that is not on that chain: it
+//                prefetches the survivor lists two frames ahead, clears the
+//                next frame's tables, stages the next frame's log-probability
+//                table and publishes its constants (survivor count, position
+//                of blank, the reciprocal the ext lanes divide with).
+//
+// A frame:
+//   P1  every candidate is evaluated once and counted in a histogram of its
+//       score (1/4 nat per bin).  The prefix merge happens here: an entry
+//       whose parent prefix is also in the beam (found through a small hash
+//       table of the beam's prefix fingerprints) adds the mass of "parent
+//       extended by last(q)" to its own pnb', takes that extension's count
+//       out of the histogram again and flags it as merged.
+//   B1
+//   P2  the histogram is scanned for the bin that holds the K-th best score
+//       (small blocks: every warp for itself, which saves a barrier).  The
+//       upper edge of the first non-empty group of bins becomes the new zero
+//       of the relative scores.
+//   P3  candidates above the cut bin take consecutive beam slots from one
+//       warp-aggregated counter and are written to the next beam, with their
+//       fingerprint entered into the next frame's hash table and, for an
+//       extension, a back-pointer node appended to the trie.  Candidates
+//       inside the cut bin are listed and, after a barrier (B3), ranked
+//       exactly among themselves (a handful).
+//   B4
 // If the cut bin is crowded (many near-equal scores) an exact radix select
-// over order-preserving integer keys replaces P3.
-// Scores are float32 relative to the best total of the previous frame; the
-// sum of the subtracted maxima is kept in float64.
+// over order-preserving integer keys replaces the list.
+//
+// Prefix identity.  A prefix is its token sequence.  Each beam entry carries
+// a 64-bit fingerprint of its sequence, fingerprint(child) =
+// mix(fingerprint(parent), token), and the fingerprint of its parent.  Two
+// candidates of a frame can name the same prefix only as "entry q stays" and
+// "q's parent, also in the beam, extends by last(q)", so the merge needs the
+// beam slot of q's parent and nothing else: a lookup of the parent's
+// fingerprint among the beam's fingerprints.  This holds no matter how often
+// a prefix has left and re-entered the beam, needs no per-prefix state in
+// HBM, and keeps the trie append-only (8 bytes per entry that enters the
+// beam).  Distinct sequences collide with probability 2^-64 per comparison.
+//
+// Scores are float32 relative to a per-frame reference within a few nats of
+// the best total; the sum of the references is kept in float64.
 #include "fltop_internal.h"
 
 namespace fltop {
 namespace {
 
 constexpr int kMaxThreads = 1024;
-constexpr int kCache = 4;          // candidate keys cached in registers per thread
-constexpr int kFastBins = 512;     // score histogram of the fast select
-constexpr float kBinsPerNat = 8.f;
+constexpr int kSmallBlock = 256;   // up to here every warp scans the histogram itself
+constexpr int kCache = 4;          // extension keys cached in registers per ext lane
+static_assert(kCache == 4, "the cached-key selects in P3 are written out for four keys");
+constexpr int kFastBins = 256;     // score histogram of the fast select
+constexpr float kBinsPerNat = 4.f;
+constexpr int kBinsPerLane = kFastBins / 32;
 constexpr int kListCap = 64;       // candidates of the cut bin ranked pairwise
 constexpr int kRadixBits = 8;      // exact fallback select
 constexpr int kBins = 1 << kRadixBits;
 constexpr int kPasses = 32 / kRadixBits;
+constexpr unsigned long long kRootPrint = 0x9E3779B97F4A7C15ull;
+constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 
-// log(exp(a) + exp(b)); symmetric in its arguments.
+// log(exp(a) + exp(b)); symmetric in its arguments.  The hardware exp2 / log2
+// approximations are used: their absolute error (about 2e-7 per call) is of the
+// order of one float32 rounding of the scores themselves.
 __device__ __forceinline__ float lse2(float a, float b) {
   const float hi = fmaxf(a, b), lo = fminf(a, b);
   if (lo == neg_inf()) return hi;
+#ifdef FLTOP_EXACT_LSE
   return hi + log1pf(expf(lo - hi));
+#else
+  return hi + __logf(1.f + __expf(lo - hi));
+#endif
 }
 
 // Order-preserving map float -> uint32 (larger float = larger key).  Key 0 is
@@ -62,14 +104,26 @@ __device__ __forceinline__ float key_score(unsigned k) {
   const unsigned u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
   return __uint_as_float(u);
 }
-// Histogram bin of a candidate: monotone in the score, bin 0 holds the best.
-__device__ __forceinline__ int score_bin(unsigned key) {
-  const int b = __float2int_rz(-key_score(key) * kBinsPerNat);
+// Histogram bin of a score: monotone, bin 0 holds the best, the last bin
+// everything below -(kFastBins-1)/kBinsPerNat.
+__device__ __forceinline__ int score_bin(float s) {
+  const int b = __float2int_rz(-s * kBinsPerNat);
   return min(kFastBins - 1, max(0, b));
 }
-// Bins are stored transposed so that the lane of warp 0 that owns bins
-// [16 l, 16 l + 16) reads them without bank conflicts.
-__device__ __forceinline__ int bin_addr(int bin) { return ((bin & 15) << 5) | (bin >> 4); }
+// Bins are stored transposed so that the lane that owns bins
+// [8 l, 8 l + 8) reads them without bank conflicts.
+__device__ __forceinline__ int bin_addr(int bin) {
+  return ((bin & (kBinsPerLane - 1)) << 5) | (bin / kBinsPerLane);
+}
+
+// Fingerprint of a prefix extended by one token.
+__device__ __forceinline__ unsigned long long child_print(unsigned long long h, int token) {
+  unsigned long long x = (h ^ (unsigned long long)(unsigned)(token + 1)) * 0x9E3779B97F4A7C15ull;
+  x ^= x >> 32;
+  x *= 0xD6E8FEB86659FD93ull;
+  x ^= x >> 32;
+  return x;
+}
 
 __device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src) {
   const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -83,59 +137,112 @@ __device__ __forceinline__ void cp_async_wait_but_one() {
   asm volatile("cp.async.wait_group 1;\n" ::: "memory");
 }
 
-// Beam fields, each a [K] array of 32-bit words, two copies (current / next).
-enum { F_NODE, F_LAST, F_PAR, F_PARNODE, F_PB, F_PNB, F_FIRST, F_LEN, F_TOT, NF };
-//   NODE     trie node id of the prefix
-//   LAST     its last token (-1 for the empty prefix)
-//   PAR      beam slot of the prefix without its last token, -1 if not in the beam
-//   PARNODE  trie node id of that parent (-1 for the empty prefix)
-//   PB, PNB  log-mass ending in blank / in the last token (relative)
-//   FIRST    head of the node's child list as of the start of the frame
-//   LEN      number of tokens
-//   TOT      lse(PB, PNB)
+// Asynchronous bulk copy shared -> global (not multicast).  A block barrier does not wait for
+// it, unlike an ordinary global store, whose acknowledgement the next barrier would sit out.
+__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, unsigned bytes) {
+  const unsigned s = (unsigned)__cvta_generic_to_shared(smem_src);
+  asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(gmem_dst),
+               "r"(s), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+}
+// All but the most recent bulk copy have read their source.
+__device__ __forceinline__ void bulk_store_wait_read_but_one() {
+  asm volatile("cp.async.bulk.wait_group.read 1;\n" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
+}
+
+// The fields of a beam entry that every candidate of the entry needs.
+struct __align__(16) Hot {
+  int last;    // last token of the prefix, -1 for the empty prefix
+  float pb;    // log-mass of alignments ending in blank (relative)
+  float pnb;   // ... ending in the last token
+  float tot;   // lse(pb, pnb)
+};
+// Identity of a beam entry.
+struct __align__(16) Ident {
+  unsigned long long print;   // fingerprint of the token sequence
+  unsigned long long pprint;  // fingerprint of the sequence without its last token
+};
+// Where a beam entry's tokens are: its trie node and its length.
+struct __align__(8) Where {
+  int node;
+  int len;
+};
+// What a frame needs to know before it starts (written by the chore warp one frame ahead).
+struct __align__(16) FrameInfo {
+  int S;           // survivors of the frame
+  int blank_j;     // position of blank among them, -1 if pruned
+  int Snb;         // non-blank survivors
+  float lp_blank;  // log-probability of blank, -inf if pruned
+  float inv_s;     // 1 / max(Snb, 1)
+  int dq, dj;      // (number of ext lanes) divmod max(Snb, 1)
+  int pad;
+};
 
 enum {
-  SC_NBEAM_NEXT = 0, SC_MAXKEY, SC_THR, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_LISTN,
-  SC_REVIVED, SC_STATUS, SC_CREATED, SC_BLANK_J0, SC_BLANK_J1,
+  // one copy per frame parity
+  SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_PER_FRAME,
+  // single copies
+  SC_THR = 2 * SC_PER_FRAME, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_TOTAL, SC_FIRST, SC_STATUS,
+  SC_CREATED,
   // exact fallback select
-  SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_COUNT
+  SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_NBEAM_NEXT, SC_COUNT
 };
+
+// Slots of the beam's fingerprint table: a power of two, at least four times the beam width
+// (twice above 1024) so that probe sequences stay short.
+__host__ __device__ inline int table_size(int K) {
+  const int want = K > 1024 ? 2 * K : 4 * K;
+  int n = 256;
+  while (n < want) n <<= 1;
+  return n;
+}
+constexpr unsigned kEmptySlot = 0xffffffffu;  // table entry: [tag : 20][beam slot : 12]
+// words of the bitmap over a frame's extension candidates (at most K * V of them)
+__host__ __device__ inline int dup_words(int K, int V) { return (K * ((V + 31) / 32) + 3) & ~3; }
+__host__ __device__ inline int node_stage_len(int K) { return (K + 1) & ~1; }
 
 // Byte offsets of the shared-memory arrays.
 struct Lay {
-  unsigned filt, sv, warp_sums, beam, newhead, st_pb, st_pnb, st_key, old2new, from, isext,
-      dirty, inbeam, lpv, hist, rhist, list_key, list_idx, scal, total;
+  unsigned sv, hot, ident, where, nstage, finfo, warp_sums, st_pb, st_pnb, st_key, dup, tab, lpv,
+      jpos, hist,
+      rhist, list_key, list_id, sel_key, sel_id, scal, total;
 };
 
 __host__ __device__ inline Lay make_layout(int K, int V) {
   Lay l;
   unsigned off = 0;
-  const unsigned W = (unsigned)(V + 31) / 32;
   auto take = [&](unsigned bytes) {
     const unsigned at = off;
-    off += (bytes + 7u) & ~7u;
+    off += (bytes + 15u) & ~15u;
     return at;
   };
-  l.filt = take(2u * K * 8);
   l.sv = take(4u * V * 8);
+  l.hot = take(2u * K * 16);
+  l.ident = take(2u * K * 16);
+  l.where = take(2u * K * 8);
+  l.nstage = take(2u * node_stage_len(K) * 8);
+  l.finfo = take(2u * 32);
   l.warp_sums = take(34 * 8);
-  l.beam = take(2u * NF * K * 4);
-  l.newhead = take(K * 4);
   l.st_pb = take(K * 4);
   l.st_pnb = take(K * 4);
   l.st_key = take(K * 4);
-  l.old2new = take(K * 4);
-  l.from = take(K * 4);
-  l.isext = take(K * 4);
-  l.dirty = take(K * 4);
-  l.inbeam = take(2u * K * W * 4);
+  l.dup = take(2u * dup_words(K, V) * 4);
+  l.tab = take(2u * table_size(K) * 4);
   l.lpv = take(2u * V * 4);
-  l.hist = take(kFastBins * 4);
+  l.jpos = take(2u * V * 4);
+  l.hist = take(2u * kFastBins * 4);
   l.rhist = take(kPasses * kBins * 4);
   l.list_key = take(kListCap * 4);
-  l.list_idx = take(kListCap * 4);
+  l.list_id = take(kListCap * 4);
+  l.sel_key = take(K * 4);
+  l.sel_id = take(K * 4);
   l.scal = take(SC_COUNT * 4);
-  l.total = (off + 15u) & ~15u;
+  l.total = off;
   return l;
 }
 
@@ -148,7 +255,7 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
   unsigned long long inc = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const unsigned long long up = __shfl_up_sync(0xffffffffu, inc, o);
+    const unsigned long long up = __shfl_up_sync(kFull, inc, o);
     if (lane >= o) inc += up;
   }
   if (lane == 31) warp_sums[warp] = inc;
@@ -158,7 +265,7 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
     unsigned long long winc = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long up = __shfl_up_sync(0xffffffffu, winc, o);
+      const unsigned long long up = __shfl_up_sync(kFull, winc, o);
       if (lane >= o) winc += up;
     }
     warp_sums[lane] = winc - w;  // exclusive prefix of each warp
@@ -169,65 +276,63 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
   return warp_sums[warp] + inc - v;
 }
 
-// Fast select, P2: warp 0 turns the score histogram into slot counters.
-// Afterwards hist[bin] holds the number of candidates in better bins, for every
-// bin up to and including the cut bin.
-__device__ __forceinline__ void scan_score_histogram(unsigned* hist, int* scal, int K) {
+// What the scan of the score histogram says about the cut.
+struct Cut {
+  int thr;        // bin that holds the K-th best score; kFastBins if everything is kept
+  int left;       // how many members of that bin are kept
+  int cut_count;  // how many are in it
+  int cut_base;   // candidates in better bins
+  int total;      // candidates altogether
+  int first;      // first lane whose group of bins is not empty (0 if there is no candidate)
+};
+
+// One warp turns the score histogram into the cut (all lanes get the result).
+__device__ __forceinline__ Cut scan_score_histogram(const unsigned* hist, int K) {
   const int lane = threadIdx.x & 31;
-  unsigned cnt[16];
+  unsigned cnt[kBinsPerLane];
   unsigned c = 0;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < kBinsPerLane; ++i) {
     cnt[i] = hist[(i << 5) | lane];
     c += cnt[i];
   }
   unsigned inc = c;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const unsigned up = __shfl_up_sync(0xffffffffu, inc, o);
+    const unsigned up = __shfl_up_sync(kFull, inc, o);
     if (lane >= o) inc += up;
   }
-  const unsigned total = __shfl_sync(0xffffffffu, inc, 31);
-  const bool all = (int)total <= K;
-  const unsigned hit = __ballot_sync(0xffffffffu, (int)inc >= K);
-  const int owner = all ? 32 : __ffs(hit) - 1;
+  Cut r;
+  const unsigned any = __ballot_sync(kFull, c != 0u);
+  r.first = any ? __ffs(any) - 1 : 0;
+  r.total = (int)__shfl_sync(kFull, inc, 31);
+  if (r.total <= K) {
+    r.thr = kFastBins; r.left = 0; r.cut_count = 0; r.cut_base = r.total;
+    return r;
+  }
+  const unsigned hit = __ballot_sync(kFull, (int)inc >= K);
+  const int owner = __ffs(hit) - 1;
   unsigned acc = inc - c;
-  if (lane < owner) {
+  int cut = 0;
+  unsigned cut_cnt = 0;
+  bool found = false;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      hist[(i << 5) | lane] = acc;
-      acc += cnt[i];
-    }
-  } else if (lane == owner) {
-    int cut = 0;
-    unsigned cut_cnt = 0;
-    bool found = false;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      if (!found) {
-        hist[(i << 5) | lane] = acc;
-        if ((int)(acc + cnt[i]) >= K) {
-          found = true;
-          cut = i;
-          cut_cnt = cnt[i];
-        } else {
-          acc += cnt[i];
-        }
+  for (int i = 0; i < kBinsPerLane; ++i) {
+    if (!found) {
+      if ((int)(acc + cnt[i]) >= K) {
+        found = true;
+        cut = i;
+        cut_cnt = cnt[i];
+      } else {
+        acc += cnt[i];
       }
     }
-    scal[SC_THR] = 16 * lane + cut;
-    scal[SC_LEFT] = K - (int)acc;      // how many of the cut bin are kept
-    scal[SC_CUT_COUNT] = (int)cut_cnt; // how many are in it
-    scal[SC_CUT_BASE] = (int)acc;      // first slot of the cut bin
-    scal[SC_NBEAM_NEXT] = K;
   }
-  if (all && lane == 0) {
-    scal[SC_THR] = kFastBins;  // no cut: every candidate is kept
-    scal[SC_LEFT] = 0;
-    scal[SC_CUT_COUNT] = 0;
-    scal[SC_CUT_BASE] = 0;
-    scal[SC_NBEAM_NEXT] = (int)total;
-  }
+  r.thr = kBinsPerLane * owner + __shfl_sync(kFull, cut, owner);
+  r.cut_base = (int)__shfl_sync(kFull, acc, owner);
+  r.cut_count = (int)__shfl_sync(kFull, cut_cnt, owner);
+  r.left = K - r.cut_base;
+  return r;
 }
 
 // Exact fallback select: after a histogram pass over one radix digit, warp 0
@@ -242,10 +347,10 @@ __device__ __forceinline__ void resolve_digit(const unsigned* h, int* scal, int 
   unsigned inc = c;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const unsigned up = __shfl_up_sync(0xffffffffu, inc, o);
+    const unsigned up = __shfl_up_sync(kFull, inc, o);
     if (lane >= o) inc += up;
   }
-  const unsigned total = __shfl_sync(0xffffffffu, inc, 31);
+  const unsigned total = __shfl_sync(kFull, inc, 31);
   if (pass == 0 && (int)total <= need) {
     if (lane == 0) {  // fewer candidates than beam slots: keep every candidate
       scal[SC_PREFIX] = 0; scal[SC_SHIFT] = 0; scal[SC_NEED] = 0; scal[SC_TAKEALL] = 0;
@@ -253,7 +358,7 @@ __device__ __forceinline__ void resolve_digit(const unsigned* h, int* scal, int 
     }
     return;
   }
-  const unsigned hit = __ballot_sync(0xffffffffu, (int)inc >= need);
+  const unsigned hit = __ballot_sync(kFull, (int)inc >= need);
   const int owner = __ffs(hit) - 1;
   if (lane == owner) {
     unsigned acc = inc - c;
@@ -274,38 +379,60 @@ __device__ __forceinline__ void resolve_digit(const unsigned* h, int* scal, int 
   }
 }
 
-__global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x;
-  const int K = p.K, V = p.V, W = (V + 31) / 32, blank = p.blank;
-  const Lay L = make_layout(K, V);
+// e divmod d for 0 <= e < 2^22 by a float reciprocal and one correction step.
+__device__ __forceinline__ void divmod_small(int e, int d, float inv_d, int& q, int& r) {
+  q = __float2int_rz(((float)e + 0.5f) * inv_d);
+  r = e - q * d;
+  if (r < 0) { --q; r += d; }
+  else if (r >= d) { ++q; r -= d; }
+}
 
-  unsigned long long* const filt_base = reinterpret_cast<unsigned long long*>(smem + L.filt);
+template <int MAXT>
+__global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
+  const int K = p.K, V = p.V, blank = p.blank;
+  const Lay L = make_layout(K, V);
+  const int TS = table_size(K);
+  const int DW = dup_words(K, V);
+  const int NSL = node_stage_len(K);
+  const unsigned tmask = (unsigned)TS - 1u;
+  const unsigned lt_mask = (1u << lane) - 1u;
+
   Survivor* const sv_base = reinterpret_cast<Survivor*>(smem + L.sv);
+  Hot* const hot_base = reinterpret_cast<Hot*>(smem + L.hot);
+  Ident* const ident_base = reinterpret_cast<Ident*>(smem + L.ident);
+  Where* const where_base = reinterpret_cast<Where*>(smem + L.where);
+  FrameInfo* const finfo = reinterpret_cast<FrameInfo*>(smem + L.finfo);
   unsigned long long* const warp_sums = reinterpret_cast<unsigned long long*>(smem + L.warp_sums);
-  int* const beam_base = reinterpret_cast<int*>(smem + L.beam);
-  int* const newhead = reinterpret_cast<int*>(smem + L.newhead);
   float* const st_pb = reinterpret_cast<float*>(smem + L.st_pb);
   float* const st_pnb = reinterpret_cast<float*>(smem + L.st_pnb);
   unsigned* const st_key = reinterpret_cast<unsigned*>(smem + L.st_key);
-  int* const old2new = reinterpret_cast<int*>(smem + L.old2new);
-  int* const from = reinterpret_cast<int*>(smem + L.from);
-  int* const isext = reinterpret_cast<int*>(smem + L.isext);
-  int* const dirty = reinterpret_cast<int*>(smem + L.dirty);
-  unsigned* const inbeam_base = reinterpret_cast<unsigned*>(smem + L.inbeam);
+  unsigned* const dup_base = reinterpret_cast<unsigned*>(smem + L.dup);
+  TrieNode* const nstage = reinterpret_cast<TrieNode*>(smem + L.nstage);
+  int* const jpos_base = reinterpret_cast<int*>(smem + L.jpos);
+  unsigned* const tab_base = reinterpret_cast<unsigned*>(smem + L.tab);
   float* const lpv_base = reinterpret_cast<float*>(smem + L.lpv);
-  unsigned* const hist = reinterpret_cast<unsigned*>(smem + L.hist);
+  unsigned* const hist_base = reinterpret_cast<unsigned*>(smem + L.hist);
   unsigned* const rhist = reinterpret_cast<unsigned*>(smem + L.rhist);
   unsigned* const list_key = reinterpret_cast<unsigned*>(smem + L.list_key);
-  int* const list_idx = reinterpret_cast<int*>(smem + L.list_idx);
+  int* const list_id = reinterpret_cast<int*>(smem + L.list_id);
+  unsigned* const sel_key = reinterpret_cast<unsigned*>(smem + L.sel_key);
+  int* const sel_id = reinterpret_cast<int*>(smem + L.sel_id);
   int* const scal = reinterpret_cast<int*>(smem + L.scal);
 
-  auto bi = [&](int buf, int f) -> int* { return beam_base + (buf * NF + f) * K; };
-  auto bf = [&](int buf, int f) -> float* { return reinterpret_cast<float*>(bi(buf, f)); };
-  auto filt = [&](int buf) -> unsigned long long* { return filt_base + buf * K; };
-  auto svbuf = [&](int t) -> Survivor* { return sv_base + (t & 3) * V; };
-  auto lpvbuf = [&](int t) -> float* { return lpv_base + (t & 1) * V; };
-  auto ibbuf = [&](int t) -> unsigned* { return inbeam_base + (t & 1) * K * W; };
+  // ---- roles -----------------------------------------------------------------------
+  const int NW = NT >> 5, warp = tid >> 5;
+  int nsw = (K + 31) >> 5;                   // stay warps: one lane per beam entry if possible
+  if (nsw > (NW - 1) / 2) nsw = (NW - 1) / 2;
+  if (nsw < 1) nsw = 1;
+  const int NS = nsw << 5;                   // stay lanes
+  const int NX = (NW - 1 - nsw) << 5;        // ext lanes
+  const bool is_chore = warp == NW - 1;
+  const bool is_stay = warp < nsw;
+  const bool is_ext = !is_chore && !is_stay;
+  const int xl = tid - NS;                   // index among the ext lanes
+  const bool warp_scans = NT <= kSmallBlock;
 
   int len = p.lengths[b];
   unsigned flags = 3u;
@@ -325,34 +452,26 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
                     : nullptr;
 
   // ---- initialise shared state -------------------------------------------------
-  for (int i = tid; i < 2 * K * W; i += NT) inbeam_base[i] = 0u;
+  for (int i = tid; i < 2 * DW; i += NT) dup_base[i] = 0u;
+  for (int i = tid; i < 2 * TS; i += NT) tab_base[i] = kEmptySlot;
   for (int i = tid; i < 2 * V; i += NT) lpv_base[i] = neg_inf();
-  for (int i = tid; i < kFastBins; i += NT) hist[i] = 0u;
-  for (int i = tid; i < K; i += NT) {
-    dirty[i] = 0;
-    old2new[i] = -1;
-  }
-  if (tid == 0) {
-    scal[SC_BLANK_J0] = -1; scal[SC_BLANK_J1] = -1;
-    scal[SC_REVIVED] = 0; scal[SC_STATUS] = 0; scal[SC_CREATED] = 0;
-    scal[SC_MAXKEY] = 0; scal[SC_LISTN] = 0;
-  }
+  for (int i = tid; i < 2 * kFastBins; i += NT) hist_base[i] = 0u;
+  if (tid < SC_COUNT) scal[tid] = 0;
   int created = 0, live_sum = 0;
   int cur = 0, nb, n_nodes, frames_seen;
   double offset;
   if (do_reset) {
     nb = bad_len && !p.streaming ? 0 : 1;
-    n_nodes = 1;
+    n_nodes = 2;  // node 0 is the empty prefix, id 1 is not used: blocks of ids start even
     offset = 0.0;
     frames_seen = 0;
     if (tid == 0) {
-      bi(0, F_NODE)[0] = 0; bi(0, F_LAST)[0] = -1; bi(0, F_PAR)[0] = -1; bi(0, F_PARNODE)[0] = -1;
-      bf(0, F_PB)[0] = 0.f; bf(0, F_PNB)[0] = neg_inf(); bi(0, F_FIRST)[0] = -1;
-      bi(0, F_LEN)[0] = 0; bf(0, F_TOT)[0] = 0.f; filt(0)[0] = 0ull;
-      TrieNode root;
-      root.parent = -1; root.token = -1; root.first_child = -1; root.next_sibling = -1;
-      root.depth = 0; root.pad = 0; root.child_filter = 0ull;
-      nodes[0] = root;
+      Hot e;
+      e.last = -1; e.pb = 0.f; e.pnb = neg_inf(); e.tot = 0.f;
+      hot_base[0] = e;
+      ident_base[0] = Ident{kRootPrint, 0ull};
+      where_base[0] = Where{0, 0};
+      nodes[0] = TrieNode{-1, -1};
     }
   } else {
     const StateHeader* hd = reinterpret_cast<const StateHeader*>(st);
@@ -360,260 +479,478 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
     status |= hd->status;
     const int32_t* a = st + kStateHeaderWords;
     for (int i = tid; i < nb; i += NT) {
-      bi(0, F_NODE)[i] = a[i]; bi(0, F_LAST)[i] = a[K + i]; bi(0, F_PAR)[i] = a[2 * K + i];
-      bi(0, F_PARNODE)[i] = a[3 * K + i];
-      const float pb = __int_as_float(a[4 * K + i]), pnb = __int_as_float(a[5 * K + i]);
-      bf(0, F_PB)[i] = pb; bf(0, F_PNB)[i] = pnb; bf(0, F_TOT)[i] = __int_as_float(a[10 * K + i]);
-      bi(0, F_FIRST)[i] = a[6 * K + i]; bi(0, F_LEN)[i] = a[7 * K + i];
-      filt(0)[i] = reinterpret_cast<const unsigned long long*>(a + 8 * K)[i];
+      Hot e;
+      e.last = a[K + i];
+      e.pb = __int_as_float(a[3 * K + i]);
+      e.pnb = __int_as_float(a[4 * K + i]);
+      e.tot = __int_as_float(a[5 * K + i]);
+      hot_base[i] = e;
+      where_base[i] = Where{a[i], a[2 * K + i]};
+      ident_base[i] = Ident{reinterpret_cast<const unsigned long long*>(a + 6 * K)[i],
+                            reinterpret_cast<const unsigned long long*>(a + 8 * K)[i]};
     }
   }
+  __syncthreads();
 
-  // ---- prologue: survivors of frames 0 and 1, log-prob table of frame 0 --------------
+  // Hash table of the beam's fingerprints.  An entry holds a beam slot and 20 bits of its
+  // fingerprint, so a probe that meets another prefix is rejected without a second load; a
+  // tag match is confirmed against the full fingerprint.  The table is never more than half
+  // full, so a probe sequence always ends at an empty entry.
+  auto table_insert = [&](unsigned* tab, unsigned long long h, int slot) {
+    const unsigned val = (((unsigned)h & 0xfffffu) << 12) | (unsigned)slot;
+    unsigned pos = (unsigned)(h >> 40) & tmask;
+    while (atomicCAS(&tab[pos], kEmptySlot, val) != kEmptySlot) pos = (pos + 1) & tmask;
+  };
+  // Beam slot of the entry with fingerprint h, or -1.
+  auto table_find = [&](const unsigned* tab, const Ident* ids, unsigned long long h) {
+    const unsigned tag = (unsigned)h & 0xfffffu;
+    unsigned pos = (unsigned)(h >> 40) & tmask;
+    while (true) {
+      const unsigned v = tab[pos];
+      if (v == kEmptySlot) return -1;
+      if ((v >> 12) == tag) {
+        const int slot = (int)(v & 0xfffu);
+        if (ids[slot].print == h) return slot;
+      }
+      pos = (pos + 1) & tmask;
+    }
+  };
+
   const int32_t* counts = p.counts + (int64_t)b * p.T;
   const Survivor* entries = p.entries + (int64_t)b * p.T * V;
-  int c0 = len > 0 ? counts[0] : 0;
-  int c1 = len > 1 ? counts[1] : 0;
-  int c2 = len > 2 ? counts[2] : 0;
-  for (int j = tid; j < c0; j += NT) cp_async8(&svbuf(0)[j], &entries[j]);
-  cp_async_commit();
-  for (int j = tid; j < c1; j += NT) cp_async8(&svbuf(1)[j], &entries[(int64_t)V + j]);
-  cp_async_commit();
-  cp_async_wait_all();
-  __syncthreads();
-  for (int j = tid; j < c0; j += NT) {
-    const Survivor s = svbuf(0)[j];
-    lpvbuf(0)[s.token] = s.logp;
-    if (s.token == blank) scal[SC_BLANK_J0] = j;
-  }
-  // in-beam child bits of a beam carried over from the previous chunk
-  for (int i = tid; i < nb; i += NT) {
-    const int par = bi(0, F_PAR)[i];
-    if (par >= 0) {
-      const int e = bi(0, F_LAST)[i];
-      atomicOr(&ibbuf(0)[par * W + (e >> 5)], 1u << (e & 31));
+  auto svbuf = [&](int t) -> Survivor* { return sv_base + (t & 3) * V; };
+  auto lpvbuf = [&](int t) -> float* { return lpv_base + (t & 1) * V; };
+
+  // Chore warp: the log-probability table and the constants of frame t1 (its survivors are
+  // in shared memory), and the table of frame t1 - 1 forgotten (t1 > 0).
+  auto stage_frame = [&](int t1, int S_prev, int S1) {
+    if (t1 > 0) {
+      float* lp_old = lpvbuf(t1 - 1);
+      const Survivor* so = svbuf(t1 - 1);
+      for (int j = lane; j < S_prev; j += 32) lp_old[so[j].token] = neg_inf();
     }
+    float* lp_new = lpvbuf(t1);
+    const Survivor* sn = svbuf(t1);
+    int bj = -1;
+    float bl = neg_inf();
+    for (int j0 = 0; j0 < S1; j0 += 32) {
+      const int j = j0 + lane;
+      bool is_blank = false;
+      float lp = neg_inf();
+      if (j < S1) {
+        const Survivor s = sn[j];
+        lp_new[s.token] = s.logp;
+        is_blank = s.token == blank;
+        lp = s.logp;
+      }
+      const unsigned m = __ballot_sync(kFull, is_blank);
+      if (m) {
+        const int src = __ffs(m) - 1;
+        bj = j0 + src;
+        bl = __shfl_sync(kFull, lp, src);
+      }
+    }
+    int* jp_new = jpos_base + (t1 & 1) * V;
+    for (int j = lane; j < S1; j += 32) jp_new[sn[j].token] = j - ((bj >= 0 && j > bj) ? 1 : 0);
+    if (lane == 0) {
+      FrameInfo f;
+      f.S = S1; f.blank_j = bj; f.Snb = S1 - (bj >= 0 ? 1 : 0); f.lp_blank = bl;
+      const int d = max(f.Snb, 1);
+      f.inv_s = 1.f / (float)d;
+      divmod_small(NX, d, f.inv_s, f.dq, f.dj);
+      f.pad = 0;
+      finfo[t1 & 1] = f;
+    }
+  };
+
+  // ---- prologue: survivors of frames 0 and 1, tables of frame 0 ----------------------
+  int c0 = 0, c1 = 0, c2 = 0;  // survivor counts of frames t, t+1, t+2 (chore warp only)
+  for (int i = tid; i < nb; i += NT) table_insert(tab_base, ident_base[i].print, i);
+  if (is_chore) {
+    c0 = len > 0 ? counts[0] : 0;
+    c1 = len > 1 ? counts[1] : 0;
+    c2 = len > 2 ? counts[2] : 0;
+    for (int j = lane; j < c0; j += 32) cp_async8(&svbuf(0)[j], &entries[j]);
+    cp_async_commit();
+    for (int j = lane; j < c1; j += 32) cp_async8(&svbuf(1)[j], &entries[(int64_t)V + j]);
+    cp_async_commit();
+    cp_async_wait_all();
+    __syncwarp();
+    stage_frame(0, 0, c0);
   }
-  int nb_prev = 0;  // size of the beam whose trie changes are still unpublished
   __syncthreads();
 
+  int pend_at = 0;
+  unsigned pend_bytes = 0u;
   for (int t = 0; t < len; ++t) {
-    const int nxt = cur ^ 1;
-    const int Scur = c0;
+    const int par = t & 1, nxt = cur ^ 1;
     const Survivor* const sv = svbuf(t);
     const float* const lpv = lpvbuf(t);
-    const unsigned* const ib = ibbuf(t);
-    int* const c_last = bi(cur, F_LAST);
-    int* const c_par = bi(cur, F_PAR);
-    float* const c_pb = bf(cur, F_PB);
-    float* const c_pnb = bf(cur, F_PNB);
-    float* const c_tot = bf(cur, F_TOT);
+    const Hot* const hc = hot_base + cur * K;
+    Hot* const hn = hot_base + nxt * K;
+    const Ident* const id_c = ident_base + cur * K;
+    Ident* const id_n = ident_base + nxt * K;
+    const Where* const wh_c = where_base + cur * K;
+    Where* const wh_n = where_base + nxt * K;
+    unsigned* const hist = hist_base + par * kFastBins;
+    unsigned* const dupbits = dup_base + par * DW;
+    const int* const jpos = jpos_base + par * V;
+    const unsigned* const tab_c = tab_base + par * TS;
+    unsigned* const tab_n = tab_base + (par ^ 1) * TS;
+    int* const sc_c = scal + par * SC_PER_FRAME;
 
-    // survivors of frame t+2 start their way to shared memory; count of frame t+3
-    if (t + 2 < len) {
-      const Survivor* src = entries + (int64_t)(t + 2) * V;
-      Survivor* dst = svbuf(t + 2);
-      for (int j = tid; j < c2; j += NT) cp_async8(&dst[j], &src[j]);
-    }
-    cp_async_commit();
-    const int c3 = (t + 3 < len) ? counts[t + 3] : 0;
+    const FrameInfo fi = finfo[par];
+    const int Snb = fi.Snb, blank_j = fi.blank_j;
+    const int Sdiv = max(Snb, 1);
+    const int next = nb * Snb;  // extension candidates of this frame
 
-    const int blank_j = scal[SC_BLANK_J0 + (t & 1)];
-    const int Snb = Scur - (blank_j >= 0 ? 1 : 0);
-    const int ncand = nb + nb * Snb;
-
-    auto ext_key = [&](int idx) -> unsigned {
-      const int e = idx - nb;
-      const int q = e / Snb;
-      int j = e - q * Snb;
-      if (blank_j >= 0 && j >= blank_j) ++j;
-      const Survivor s = sv[j];
-      if ((ib[q * W + (s.token >> 5)] >> (s.token & 31)) & 1u) return 0u;  // merged into a stay
-      const float base = (s.token == c_last[q]) ? c_pb[q] : c_tot[q];
-      return score_key(base + s.logp);
+    // position of the j-th non-blank survivor in the survivor list
+    const int blank_at = blank_j >= 0 ? blank_j : 0x7fffffff;
+    auto sv_index = [&](int j) -> int { return j + (j >= blank_at ? 1 : 0); };
+    // score of entry e extended by non-blank survivor j
+    auto ext_score = [&](const Hot& e, int j) -> float {
+      const Survivor s = sv[sv_index(j)];
+      return ((s.token == e.last) ? e.pb : e.tot) + s.logp;
     };
-    auto stay_key = [&](int i) -> unsigned {
-      const int e = c_last[i];
-      const float npb = c_tot[i] + lpv[blank];
+    auto ext_key = [&](const Hot& e, int j) -> unsigned { return score_key(ext_score(e, j)); };
+    auto ext_token = [&](int j) -> int { return sv[sv_index(j)].token; };
+    // extension candidate e = q * Snb + j names a prefix that is already in the beam
+    auto merged = [&](int e) -> bool { return (dupbits[e >> 5] >> (e & 31)) & 1u; };
+    auto count = [&](float score) { atomicAdd(&hist[bin_addr(score_bin(score))], 1u); };
+    // stay candidate of entry q, including the prefix merge
+    auto stay_eval = [&](int q) -> unsigned {
+      const Hot e = hc[q];
+      const float npb = e.tot + fi.lp_blank;
       float npnb = neg_inf();
-      if (e >= 0) {
-        const float le = lpv[e];
-        npnb = c_pnb[i] + le;
-        const int par = c_par[i];
-        if (par >= 0) {
-          const float base = (c_last[par] == e) ? c_pb[par] : c_tot[par];
-          npnb = lse2(npnb, base + le);
+      if (e.last >= 0) {
+        const float le = lpv[e.last];
+        npnb = e.pnb + le;
+        const int pq = table_find(tab_c, id_c, id_c[q].pprint);
+        if (pq >= 0) {
+          const Hot pe = hc[pq];
+          const float dup = ((pe.last == e.last) ? pe.pb : pe.tot) + le;
+          if (dup != neg_inf()) {  // the parent's extension by last(q) names this prefix
+            npnb = lse2(npnb, dup);
+            atomicSub(&hist[bin_addr(score_bin(dup))], 1u);
+            const int ed = pq * Snb + jpos[e.last];
+            atomicOr(&dupbits[ed >> 5], 1u << (ed & 31));
+          }
         }
       }
-      st_pb[i] = npb;
-      st_pnb[i] = npnb;
-      const unsigned key = score_key(lse2(npb, npnb));
-      st_key[i] = key;
+      st_pb[q] = npb;
+      st_pnb[q] = npnb;
+      const float tot = lse2(npb, npnb);
+      const unsigned key = score_key(tot);
+      st_key[q] = key;
+      if (key) count(tot);
       return key;
     };
-    auto cand_key = [&](int idx) -> unsigned { return idx < nb ? st_key[idx] : ext_key(idx); };
-
-    // ---- P1: evaluate every candidate once, score histogram, running maximum ----------
-    unsigned kc[kCache];
-    {
-      unsigned local_max = 0u;
-#pragma unroll
-      for (int k = 0; k < kCache; ++k) {
-        const int idx = tid + k * NT;
-        unsigned key = 0u;
-        if (idx < ncand) key = idx < nb ? stay_key(idx) : ext_key(idx);
-        kc[k] = key;
-        if (key) atomicAdd(&hist[bin_addr(score_bin(key))], 1u);
-        local_max = max(local_max, key);
-      }
-      for (int idx = tid + kCache * NT; idx < ncand; idx += NT) {
-        const unsigned key = idx < nb ? stay_key(idx) : ext_key(idx);
-        if (key) atomicAdd(&hist[bin_addr(score_bin(key))], 1u);
-        local_max = max(local_max, key);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1)
-        local_max = max(local_max, __shfl_xor_sync(0xffffffffu, local_max, o));
-      if ((tid & 31) == 0 && local_max)
-        atomicMax(reinterpret_cast<unsigned*>(&scal[SC_MAXKEY]), local_max);
-      if (tid == 0) scal[SC_BLANK_J0 + ((t + 1) & 1)] = -1;
-    }
-    cp_async_wait_but_one();  // survivors of frame t+1 have landed (this thread's part)
-    __syncthreads();          // B1
-
-    // ---- P2: warp 0 finds the cut; the others do the bookkeeping ------------------------
-    if (tid < 32) {
-      scan_score_histogram(hist, scal, K);
-    } else {
-      // publish the child lists changed last frame: to HBM and to the surviving entry
-      const int o = cur ^ 1;  // last frame's beam
-      const int n_pub = max(nb_prev, nb);
-      if (tid == 32) scal[SC_REVIVED] = 0;
-      for (int i = tid - 32; i < n_pub; i += NT - 32) {
-        if (i < nb_prev && dirty[i]) {
-          dirty[i] = 0;
-          const int head = newhead[i];
-          const unsigned long long f = filt(o)[i];
-          TrieNode* n = &nodes[bi(o, F_NODE)[i]];
-          n->first_child = head;
-          n->child_filter = f;
-          const int s = old2new[i];
-          if (s >= 0) {
-            bi(cur, F_FIRST)[s] = head;
-            filt(cur)[s] = f;
-          }
-        }
-        old2new[i] = -1;  // from here on: slot of current entry i in the next beam
-      }
-      // log-prob table: forget frame t, stage frame t+1
-      float* lp_now = lpvbuf(t);
-      for (int j = tid - 32; j < Scur; j += NT - 32) lp_now[sv[j].token] = neg_inf();
-      if (t + 1 < len) {
-        float* lp_next = lpvbuf(t + 1);
-        const Survivor* sn = svbuf(t + 1);
-        for (int j = tid - 32; j < c1; j += NT - 32) {
-          const Survivor s = sn[j];
-          lp_next[s.token] = s.logp;
-          if (s.token == blank) scal[SC_BLANK_J0 + ((t + 1) & 1)] = j;
-        }
-      }
-    }
-    __syncthreads();  // B2
-
-    // ---- P3: selected candidates take their slots in the next beam ---------------------
-    const int thr = scal[SC_THR], left = scal[SC_LEFT];
-    const int cut_count = scal[SC_CUT_COUNT], cut_base = scal[SC_CUT_BASE];
-    const unsigned maxkey = (unsigned)scal[SC_MAXKEY];
-    const int nbn = maxkey ? scal[SC_NBEAM_NEXT] : 0;
-    const float best = maxkey ? key_score(maxkey) : 0.f;
-    const bool take_all = cut_count == left;  // also true when there is no cut at all
-    const bool use_list = !take_all && cut_count <= kListCap;
-
-    auto place = [&](int idx, unsigned key, int slot) {
-      if (idx < nb) {
-        old2new[idx] = slot;
-        bi(nxt, F_NODE)[slot] = bi(cur, F_NODE)[idx];
-        bi(nxt, F_LAST)[slot] = c_last[idx];
-        bi(nxt, F_PARNODE)[slot] = bi(cur, F_PARNODE)[idx];
-        bf(nxt, F_PB)[slot] = st_pb[idx] - best;
-        bf(nxt, F_PNB)[slot] = st_pnb[idx] - best;
-        bf(nxt, F_TOT)[slot] = key_score(key) - best;
-        bi(nxt, F_FIRST)[slot] = bi(cur, F_FIRST)[idx];
-        bi(nxt, F_LEN)[slot] = bi(cur, F_LEN)[idx];
-        filt(nxt)[slot] = filt(cur)[idx];
-        from[slot] = idx;
-        isext[slot] = 0;
-      } else {
-        const int e = idx - nb;
-        const int q = e / Snb;
-        int j = e - q * Snb;
-        if (blank_j >= 0 && j >= blank_j) ++j;
-        const float sc = key_score(key) - best;
-        bi(nxt, F_NODE)[slot] = -1;
-        bi(nxt, F_LAST)[slot] = sv[j].token;
-        bi(nxt, F_PARNODE)[slot] = bi(cur, F_NODE)[q];
-        bf(nxt, F_PB)[slot] = neg_inf();
-        bf(nxt, F_PNB)[slot] = sc;
-        bf(nxt, F_TOT)[slot] = sc;
-        bi(nxt, F_FIRST)[slot] = -1;
-        bi(nxt, F_LEN)[slot] = bi(cur, F_LEN)[q] + 1;
-        filt(nxt)[slot] = 0ull;
-        from[slot] = q;
-        isext[slot] = 1;
-      }
+    // this lane's extension candidates: e_first, e_first + NX, ... as (q, j) pairs
+    int q0 = 0, j0 = 0;
+    auto step = [&](int& q, int& j) {
+      q += fi.dq;
+      j += fi.dj;
+      if (j >= Sdiv) { j -= Sdiv; ++q; }
+    };
+    // (q, j) of this lane's k-th extension candidate
+    auto nth = [&](int k, int& q, int& j) {
+      q = q0 + k * fi.dq;
+      j = j0 + k * fi.dj;
+      while (j >= Sdiv) { j -= Sdiv; ++q; }
     };
 
-    for (int i = tid; i < nb; i += NT) newhead[i] = bi(cur, F_FIRST)[i];
-
-    if (take_all || use_list) {
-      auto assign = [&](int idx, unsigned key) {
-        if (!key) return;
-        const int bin = score_bin(key);
-        if (bin < thr || (bin == thr && take_all)) {
-          place(idx, key, (int)atomicAdd(&hist[bin_addr(bin)], 1u));
-        } else if (bin == thr) {
-          const int li = atomicAdd(&scal[SC_LISTN], 1);
-          list_key[li] = key;
-          list_idx[li] = idx;
-        }
-      };
+    // ---- P1: every candidate is evaluated once and counted -----------------------------
+    unsigned kc[kCache];
+    unsigned kstay = 0u;
+#pragma unroll
+    for (int k = 0; k < kCache; ++k) kc[k] = 0u;
+    if (is_stay) {
+      if (tid < nb) kstay = stay_eval(tid);
+      for (int i = tid + NS; i < nb; i += NS) stay_eval(i);
+    } else if (is_ext) {
+      divmod_small(xl, Sdiv, fi.inv_s, q0, j0);
+      int q = q0, j = j0;
 #pragma unroll
       for (int k = 0; k < kCache; ++k) {
-        const int idx = tid + k * NT;
-        if (idx < ncand) assign(idx, kc[k]);
+        if (xl + k * NX < next) {
+          const float sc = ext_score(hc[q], j);
+          step(q, j);
+          kc[k] = score_key(sc);
+          if (sc != neg_inf()) count(sc);
+        }
       }
-      for (int idx = tid + kCache * NT; idx < ncand; idx += NT) assign(idx, cand_key(idx));
-      if (!take_all) {
-        __syncthreads();  // B3: the cut bin's members are listed
-        // exact order inside the cut bin: score, then candidate index
-        for (int li = tid; li < cut_count; li += NT) {
-          const unsigned key = list_key[li];
-          const int idx = list_idx[li];
-          int rank = 0;
-          for (int j = 0; j < cut_count; ++j) {
-            const unsigned kj = list_key[j];
-            rank += (kj > key || (kj == key && list_idx[j] < idx)) ? 1 : 0;
+      for (int e = xl + kCache * NX; e < next; e += NX) {
+        const float sc = ext_score(hc[q], j);
+        step(q, j);
+        if (sc != neg_inf()) count(sc);
+      }
+    } else {
+      // chore warp: the nodes staged by frame t-1 go to the trie, survivors of frame t+2 start
+      // their way to shared memory, the tables of frame t+1 start empty
+      if (lane == 0 && pend_bytes) {
+        bulk_store(nodes + pend_at, nstage + (par ^ 1) * NSL, pend_bytes);
+        bulk_store_wait_read_but_one();  // the staging buffer of this frame is free again
+      }
+      if (t + 2 < len) {
+        const Survivor* src = entries + (int64_t)(t + 2) * V;
+        Survivor* dst = svbuf(t + 2);
+        for (int j = lane; j < c2; j += 32) cp_async8(&dst[j], &src[j]);
+      }
+      cp_async_commit();
+      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+      const uint4 ones = make_uint4(~0u, ~0u, ~0u, ~0u);
+      uint4* hist_n = reinterpret_cast<uint4*>(hist_base + (par ^ 1) * kFastBins);
+      uint4* dup_n = reinterpret_cast<uint4*>(dup_base + (par ^ 1) * DW);
+      uint4* tb_n = reinterpret_cast<uint4*>(tab_n);
+      for (int i = lane; i < kFastBins / 4; i += 32) hist_n[i] = zero;
+      for (int i = lane; i < DW / 4; i += 32) dup_n[i] = zero;
+      for (int i = lane; i < TS / 4; i += 32) tb_n[i] = ones;
+      if (lane == 0) {
+        int* sc_n = scal + (par ^ 1) * SC_PER_FRAME;
+        sc_n[SC_LISTN] = 0;
+        sc_n[SC_SLOT] = 0;
+        sc_n[SC_SLOT_E] = 0;
+      }
+    }
+    __syncthreads();  // B1
+
+    // ---- P2: the cut -------------------------------------------------------------------
+    // The chore warp does not scan: while the others do, it stages the log-prob table and
+    // the constants of frame t+1 (and fetches the survivor count of frame t+3); it takes
+    // the cut from warp 0.
+    auto chore_between = [&]() {
+      const int c3 = (t + 3 < len) ? counts[t + 3] : 0;
+      cp_async_wait_but_one();  // survivors of frame t+1 have landed
+      __syncwarp();
+      if (t + 1 < len) stage_frame(t + 1, c0, c1);
+      c0 = c1; c1 = c2; c2 = c3;
+    };
+    auto publish_cut = [&](const Cut& c) {
+      scal[SC_THR] = c.thr; scal[SC_LEFT] = c.left; scal[SC_CUT_COUNT] = c.cut_count;
+      scal[SC_CUT_BASE] = c.cut_base; scal[SC_TOTAL] = c.total; scal[SC_FIRST] = c.first;
+    };
+    auto read_cut = [&](Cut& c) {
+      c.thr = scal[SC_THR]; c.left = scal[SC_LEFT]; c.cut_count = scal[SC_CUT_COUNT];
+      c.cut_base = scal[SC_CUT_BASE]; c.total = scal[SC_TOTAL]; c.first = scal[SC_FIRST];
+    };
+    Cut cut;
+    if (warp_scans) {
+      if (!is_chore) {
+        cut = scan_score_histogram(hist, K);
+        if (warp == 0) {
+          if (lane == 0) publish_cut(cut);
+          __threadfence_block();
+          asm volatile("bar.arrive 1, 64;" ::: "memory");  // releases the chore warp
+        }
+      } else {
+        chore_between();
+        asm volatile("bar.sync 1, 64;" ::: "memory");      // warp 0 has published the cut
+        read_cut(cut);
+      }
+    } else {
+      if (warp == 0) {
+        cut = scan_score_histogram(hist, K);
+        if (lane == 0) publish_cut(cut);
+      } else if (is_chore) {
+        chore_between();
+      }
+      __syncthreads();  // B2 (large blocks only)
+      read_cut(cut);
+    }
+    // new zero of the relative scores: the upper edge of the first non-empty group of bins
+    const float best = -(float)(cut.first * kBinsPerLane) * (1.f / kBinsPerNat);
+    const bool take_all = cut.cut_count == cut.left;  // also true when there is no cut at all
+    const bool use_list = !take_all && cut.cut_count <= kListCap;
+    int nbn = min(cut.total, K);
+    TrieNode* const nst = nstage + par * NSL;
+    // the frame's nodes get ids n_nodes .. n_nodes + nbn - 1 (the slots of stays stay unused)
+    const bool arena_ok = (int64_t)n_nodes + NSL <= p.nodes_per_utt;
+
+    // ---- P3: selected candidates take their slots in the next beam ---------------------
+    auto place_stay = [&](int q, unsigned key, int slot) {
+      if ((unsigned)slot >= (unsigned)K) return;  // only reachable with NaN scores
+      Hot e;
+      e.last = hc[q].last;
+      e.pb = st_pb[q] - best;
+      e.pnb = st_pnb[q] - best;
+      e.tot = key_score(key) - best;
+      hn[slot] = e;
+      const Ident id = id_c[q];
+      id_n[slot] = id;
+      wh_n[slot] = wh_c[q];
+      table_insert(tab_n, id.print, slot);
+    };
+    auto place_ext = [&](int q, int tok, unsigned key, int slot) {
+      if ((unsigned)slot >= (unsigned)K) return;
+      const float sc = key_score(key) - best;
+      Hot e;
+      e.last = tok; e.pb = neg_inf(); e.pnb = sc; e.tot = sc;
+      hn[slot] = e;
+      const unsigned long long hp = id_c[q].print;
+      const unsigned long long h = child_print(hp, tok);
+      id_n[slot] = Ident{h, hp};
+      table_insert(tab_n, h, slot);
+      const Where w = wh_c[q];
+      // back-pointer node: staged here, written to the trie in one piece after the frame
+      nst[slot] = TrieNode{w.node, tok};
+      ++created;
+      wh_n[slot] = Where{arena_ok ? n_nodes + slot : 0, w.len + 1};
+    };
+    // a candidate by its id: beam entry in the high half, 0 (stay) or j + 1 (extension by the
+    // j-th non-blank survivor) in the low half
+    auto place_by_id = [&](int id, unsigned key, int slot) {
+      const int q = id >> 16, j1 = id & 0xffff;
+      if (j1 == 0) place_stay(q, key, slot);
+      else place_ext(q, ext_token(j1 - 1), key, slot);
+    };
+
+    if (take_all || use_list) {
+      // key thresholds of the cut: key > k_hi is above the cut bin, key > k_lo is in it or above
+      const unsigned k_lo = (cut.thr >= kFastBins - 1)
+                                ? 0u
+                                : score_key(-(float)(cut.thr + 1) * (1.f / kBinsPerNat));
+      const unsigned k_hi = take_all ? k_lo
+                                     : (cut.thr == 0 ? 0xffffffffu
+                                                     : score_key(-(float)cut.thr * (1.f / kBinsPerNat)));
+      // P3a: every candidate above the cut bin takes a beam slot and is noted there; stays
+      // fill the beam from slot 0 upwards, extensions from the last slot downwards.
+      auto list_add = [&](unsigned key, int id) {
+        const int li = atomicAdd(&sc_c[SC_LISTN], 1);
+        if (li < kListCap) {
+          list_key[li] = key;
+          list_id[li] = id;
+        }
+      };
+      if (is_stay) {
+        for (int base = 0; base < nb || base == 0; base += NS) {
+          const int i = base + tid;
+          const unsigned key = base == 0 ? kstay : (i < nb ? st_key[i] : 0u);
+          const bool sel = key > k_hi;
+          const unsigned m = __ballot_sync(kFull, sel);
+          if (m) {
+            int at = 0;
+            if (lane == 0) at = atomicAdd(&sc_c[SC_SLOT], __popc(m));
+            at = __shfl_sync(kFull, at, 0) + __popc(m & lt_mask);
+            if (sel && at < K) {
+              sel_key[at] = key;
+              sel_id[at] = i << 16;
+            }
           }
-          if (rank < left) place(idx, key, cut_base + rank);
+          if (!sel && key > k_lo) list_add(key, i << 16);
+        }
+      } else if (is_ext) {
+        // `n` consecutive places for this lane, n <= 7 (warp-collective)
+        auto claim = [&](int n) -> int {
+          const unsigned b0 = __ballot_sync(kFull, n & 1);
+          const unsigned b1 = __ballot_sync(kFull, n & 2);
+          const unsigned b2 = __ballot_sync(kFull, n & 4);
+          if (!(b0 | b1 | b2)) return 0;
+          int at = 0;
+          if (lane == 0)
+            at = atomicAdd(&sc_c[SC_SLOT_E], __popc(b0) + 2 * __popc(b1) + 4 * __popc(b2));
+          at = __shfl_sync(kFull, at, 0);
+          return at + __popc(b0 & lt_mask) + 2 * __popc(b1 & lt_mask) + 4 * __popc(b2 & lt_mask);
+        };
+        auto note = [&](int at, unsigned key, int id) {
+          const int slot = nbn - 1 - at;
+          if ((unsigned)slot < (unsigned)K) {
+            sel_key[slot] = key;
+            sel_id[slot] = id;
+          }
+        };
+        // cached candidates: settle which are selected, then take the places in one go
+        unsigned want = 0u;  // bit k: cached candidate k is in the cut bin or above
+#pragma unroll
+        for (int k = 0; k < kCache; ++k) want |= (kc[k] > k_lo ? 1u : 0u) << k;
+        unsigned selm = 0u;
+        int ids[kCache];
+#pragma unroll
+        for (int k = 0; k < kCache; ++k) ids[k] = 0;
+        for (unsigned m = want; m; m &= m - 1) {
+          const int k = __ffs(m) - 1;
+          if (merged(xl + k * NX)) continue;
+          const unsigned key = k == 0 ? kc[0] : k == 1 ? kc[1] : k == 2 ? kc[2] : kc[3];
+          int q, j;
+          nth(k, q, j);
+          const int id = (q << 16) | (j + 1);
+          if (key > k_hi) {
+            selm |= 1u << k;
+            if (k == 0) ids[0] = id; else if (k == 1) ids[1] = id; else if (k == 2) ids[2] = id; else ids[3] = id;
+          } else {
+            list_add(key, id);
+          }
+        }
+        int at = claim(__popc(selm));
+#pragma unroll
+        for (int k = 0; k < kCache; ++k)
+          if ((selm >> k) & 1u) note(at++, kc[k], ids[k]);
+        // candidates beyond the cache are evaluated again
+        int q, j;
+        nth(kCache, q, j);
+        for (int base = kCache * NX; base < next; base += NX) {
+          unsigned key = (xl + base < next) ? ext_key(hc[q], j) : 0u;
+          if (key > k_lo && merged(xl + base)) key = 0u;
+          const bool sel = key > k_hi;
+          const int a1 = claim(sel ? 1 : 0);
+          if (sel) note(a1, key, (q << 16) | (j + 1));
+          else if (key > k_lo) list_add(key, (q << 16) | (j + 1));
+          step(q, j);
+        }
+      }
+      __syncthreads();  // B3: every selected candidate is noted, the cut bin's members listed
+      // P3b: one candidate per lane is written to the next beam; the chore warp meanwhile
+      // ranks the members of the cut bin exactly (score, then candidate id) and writes the
+      // winners to the slots between the stays and the extensions.
+      const int n_stay = min(sc_c[SC_SLOT], K);
+      if (is_stay) {
+        for (int s2 = tid; s2 < n_stay; s2 += NS) place_stay(sel_id[s2] >> 16, sel_key[s2], s2);
+      } else if (is_ext) {
+        const int n_ext = min(sc_c[SC_SLOT_E], K);
+        for (int x = xl; x < n_ext; x += NX) {
+          const int slot = nbn - 1 - x;
+          if (slot >= 0) place_by_id(sel_id[slot], sel_key[slot], slot);
+        }
+      } else if (!take_all) {
+        for (int li = lane; li < cut.cut_count; li += 32) {
+          const unsigned key = list_key[li];
+          const int id = list_id[li];
+          int rank = 0;
+          for (int j = 0; j < cut.cut_count; ++j) {
+            const unsigned kj = list_key[j];
+            rank += (kj > key || (kj == key && list_id[j] < id)) ? 1 : 0;
+          }
+          if (rank < cut.left) place_by_id(id, key, n_stay + rank);
         }
       }
     } else {
       // ---- exact fallback: radix select over the integer keys ------------------------
+      auto for_each_candidate = [&](auto&& f) {
+        if (is_stay) {
+          for (int i = tid; i < nb; i += NS) f(st_key[i], i << 16);
+        } else if (is_ext) {
+          int q = q0, j = j0;
+          for (int e = xl; e < next; e += NX) {
+            unsigned key = ext_key(hc[q], j);
+            if (key && merged(e)) key = 0u;
+            f(key, (q << 16) | (j + 1));
+            step(q, j);
+          }
+        }
+      };
       for (int i = tid; i < kPasses * kBins; i += NT) rhist[i] = 0u;
       if (tid == 0) {
         scal[SC_PREFIX] = 0; scal[SC_NEED] = K; scal[SC_DONE] = 0; scal[SC_TAKEALL] = 0;
-        scal[SC_SHIFT] = 0;
+        scal[SC_SHIFT] = 0; scal[SC_NBEAM_NEXT] = K;
       }
       __syncthreads();
       for (int pass = 0; pass < kPasses; ++pass) {
         const int sh = 32 - kRadixBits * (pass + 1);
         const unsigned prefix = (unsigned)scal[SC_PREFIX];
         unsigned* h = rhist + pass * kBins;
-        for (int idx = tid; idx < ncand; idx += NT) {
-          const unsigned key = cand_key(idx);
+        for_each_candidate([&](unsigned key, int) {
           if (key && (pass == 0 || (key >> (sh + kRadixBits)) == prefix))
             atomicAdd(&h[(key >> sh) & (kBins - 1)], 1u);
-        }
+        });
         __syncthreads();
         if (tid < 32) resolve_digit(h, scal, pass, sh);
         __syncthreads();
@@ -623,140 +960,52 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
       const unsigned prefix = (unsigned)scal[SC_PREFIX];
       const int need = scal[SC_NEED];
       const bool r_all = scal[SC_TAKEALL] != 0;
+      nbn = scal[SC_NBEAM_NEXT];
       unsigned long long mine = 0ull;
-      for (int idx = tid; idx < ncand; idx += NT) {
-        const unsigned key = cand_key(idx);
+      for_each_candidate([&](unsigned key, int) {
         if (key) {
           const unsigned hk = key >> sh;
           mine += (hk > prefix) ? 1ull : ((hk == prefix) ? (1ull << 32) : 0ull);
         }
-      }
+      });
       unsigned long long total;
       const unsigned long long excl = block_exclusive_scan(mine, warp_sums, &total);
       int gt_rank = (int)(excl & 0xffffffffull), eq_rank = (int)(excl >> 32);
       const int total_gt = (int)(total & 0xffffffffull);
-      for (int idx = tid; idx < ncand; idx += NT) {
-        const unsigned key = cand_key(idx);
-        if (!key) continue;
+      for_each_candidate([&](unsigned key, int id) {
+        if (!key) return;
         const unsigned hk = key >> sh;
+        int slot = -1;
         if (hk > prefix) {
-          place(idx, key, gt_rank++);
+          slot = gt_rank++;
         } else if (hk == prefix) {
-          if (r_all || eq_rank < need) place(idx, key, total_gt + eq_rank);
+          if (r_all || eq_rank < need) slot = total_gt + eq_rank;
           ++eq_rank;
         }
-      }
+        if (slot >= 0) place_by_id(id, key, slot);
+      });
     }
-    __syncthreads();  // B4: the next beam is complete except for node ids and parent slots
-
-    // ---- P5: trie nodes, parent slots, in-beam child bits of the next frame ------------
-    unsigned* const ib_next = ibbuf(t + 1);
-    for (int s = tid; s < nbn; s += NT) {
-      const int q = from[s];
-      const int tok = bi(nxt, F_LAST)[s];
-      int par;
-      if (isext[s]) {
-        par = old2new[q];
-        int node = -1;
-        if ((filt(cur)[q] >> (tok & 63)) & 1ull) {
-          // a child with this filter bit exists: walk the parent's child list
-          int id = bi(cur, F_FIRST)[q];
-          for (int it = 0; id >= 0 && it <= V; ++it) {
-            const int4 rec = *reinterpret_cast<const int4*>(&nodes[id]);  // parent, token, first, next
-            if (rec.y == tok) {
-              node = id;
-              bi(nxt, F_FIRST)[s] = rec.z;
-              filt(nxt)[s] = nodes[id].child_filter;
-              scal[SC_REVIVED] = 1;
-              break;
-            }
-            id = rec.w;
-          }
-        }
-        if (node < 0) {
-          const int id = n_nodes + s;
-          if (id < p.nodes_per_utt) {
-            const int prev = atomicExch(&newhead[q], id);
-            atomicOr(&filt(cur)[q], 1ull << (tok & 63));
-            dirty[q] = 1;
-            TrieNode n;
-            n.parent = bi(cur, F_NODE)[q]; n.token = tok; n.first_child = -1;
-            n.next_sibling = prev; n.depth = bi(nxt, F_LEN)[s]; n.pad = 0; n.child_filter = 0ull;
-            nodes[id] = n;
-            node = id;
-            ++created;
-          } else {
-            node = 0;
-            scal[SC_STATUS] = 2;  // FLTOP_ST_ARENA_FULL
-          }
-        }
-        bi(nxt, F_NODE)[s] = node;
-      } else {
-        const int op = c_par[q];
-        par = op >= 0 ? old2new[op] : -1;
-      }
-      bi(nxt, F_PAR)[s] = par;
-      if (par >= 0) atomicOr(&ib_next[par * W + (tok >> 5)], 1u << (tok & 31));
-    }
-    {
-      unsigned* const ib_now = ibbuf(t);
-      for (int i = tid; i < nb; i += NT) {
-        const int par = c_par[i];
-        if (par >= 0) ib_now[par * W + (c_last[i] >> 5)] = 0u;
-      }
-    }
-    for (int i = tid; i < kFastBins; i += NT) hist[i] = 0u;
-    if (tid == 0) {
-      scal[SC_MAXKEY] = 0;
-      scal[SC_LISTN] = 0;
-    }
-    if (!maxkey) status |= 8;  // FLTOP_ST_EMPTY_BEAM
+    if (cut.total == 0) status |= 8;  // FLTOP_ST_EMPTY_BEAM
     offset += (double)best;
-    __syncthreads();  // B5
+    __syncthreads();  // B4: the next beam and its hash table are complete
 
-    if (scal[SC_REVIVED]) {
-      // a prefix came back into the beam: entries that extend it find their parent again
-      for (int s = tid; s < nbn; s += NT) {
-        if (isext[s] && bi(nxt, F_NODE)[s] < n_nodes) {
-          const int x = bi(nxt, F_NODE)[s];
-          for (int s2 = 0; s2 < nbn; ++s2) {
-            if (bi(nxt, F_PARNODE)[s2] == x && bi(nxt, F_PAR)[s2] != s) {
-              bi(nxt, F_PAR)[s2] = s;
-              const int tk = bi(nxt, F_LAST)[s2];
-              atomicOr(&ib_next[s * W + (tk >> 5)], 1u << (tk & 31));
-            }
-          }
-        }
-      }
-      __syncthreads();
-    }
-    n_nodes += nbn;
+    // (chore warp) what the next frame has to write out
+    pend_at = n_nodes;
+    pend_bytes = (arena_ok && nbn > 0) ? (unsigned)(((nbn + 1) & ~1) * sizeof(TrieNode)) : 0u;
+    if (!arena_ok && nbn > 0) status |= 2;  // FLTOP_ST_ARENA_FULL
+    n_nodes += (nbn + 1) & ~1;
     live_sum += nbn;
-    nb_prev = nb;
     nb = nbn;
     cur = nxt;
-    c0 = c1; c1 = c2; c2 = c3;
   }
   frames_seen += len;
-
-  // trie changes of the last frame
-  for (int i = tid; i < nb_prev; i += NT) {
-    if (dirty[i]) {
-      dirty[i] = 0;
-      const int o = cur ^ 1;
-      const int head = newhead[i];
-      const unsigned long long f = filt(o)[i];
-      TrieNode* n = &nodes[bi(o, F_NODE)[i]];
-      n->first_child = head;
-      n->child_filter = f;
-      const int s = old2new[i];
-      if (s >= 0) {
-        bi(cur, F_FIRST)[s] = head;
-        filt(cur)[s] = f;
-      }
-    }
+  // the last frame's nodes; the read-out below walks the trie, so wait for all of them
+  if (is_chore && lane == 0) {
+    if (pend_bytes) bulk_store(nodes + pend_at, nstage + ((len - 1) & 1) * NSL, pend_bytes);
+    bulk_store_wait_all();
   }
   __syncthreads();
+
   status |= scal[SC_STATUS];
   if (p.stats) {
     if (created) atomicAdd(&scal[SC_CREATED], created);
@@ -767,16 +1016,22 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
     }
   }
 
+  const Hot* const hc = hot_base + cur * K;
+  const Ident* const id_c = ident_base + cur * K;
+  const Where* const wh_c = where_base + cur * K;
+
   // ---- keep the beam for the next chunk (streaming) -----------------------------------
   if (p.streaming) {
     int32_t* a = st + kStateHeaderWords;
     for (int i = tid; i < nb; i += NT) {
-      a[i] = bi(cur, F_NODE)[i]; a[K + i] = bi(cur, F_LAST)[i]; a[2 * K + i] = bi(cur, F_PAR)[i];
-      a[3 * K + i] = bi(cur, F_PARNODE)[i];
-      a[4 * K + i] = bi(cur, F_PB)[i]; a[5 * K + i] = bi(cur, F_PNB)[i];
-      a[6 * K + i] = bi(cur, F_FIRST)[i]; a[7 * K + i] = bi(cur, F_LEN)[i];
-      reinterpret_cast<unsigned long long*>(a + 8 * K)[i] = filt(cur)[i];
-      a[10 * K + i] = bi(cur, F_TOT)[i];
+      const Hot e = hc[i];
+      const Where w = wh_c[i];
+      const Ident id = id_c[i];
+      a[i] = w.node; a[K + i] = e.last; a[2 * K + i] = w.len;
+      a[3 * K + i] = __float_as_int(e.pb); a[4 * K + i] = __float_as_int(e.pnb);
+      a[5 * K + i] = __float_as_int(e.tot);
+      reinterpret_cast<unsigned long long*>(a + 6 * K)[i] = id.print;
+      reinterpret_cast<unsigned long long*>(a + 8 * K)[i] = id.pprint;
     }
     if (tid == 0) {
       StateHeader* hd = reinterpret_cast<StateHeader*>(st);
@@ -789,22 +1044,22 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
   // ---- hypotheses, best first (GetHighestScorePrefix over the whole beam) ----------
   if (do_emit) {
     const int Lout = p.L;
-    const float* tot = bf(cur, F_TOT);
     bool truncated = false;
     for (int i = tid; i < nb; i += NT) {
-      const float ti = tot[i];
+      const float ti = hc[i].tot;
       int rank = 0;
       for (int j = 0; j < nb; ++j) {
-        const float tj = tot[j];
+        const float tj = hc[j].tot;
         rank += (tj > ti || (tj == ti && j < i)) ? 1 : 0;
       }
       const int64_t o = (int64_t)b * K + rank;
       p.out_scores[o] = (float)(offset + (double)ti);
-      const int n = bi(cur, F_LEN)[i];
+      const Where w = wh_c[i];
+      const int n = w.len;
       p.out_lens[o] = n;
       if (n > Lout) truncated = true;
       int32_t* dst = p.out_tokens + o * Lout;
-      int node = bi(cur, F_NODE)[i];
+      int node = w.node;
       for (int d = n - 1; d >= 0 && node > 0; --d) {
         const int2 rec = *reinterpret_cast<const int2*>(&nodes[node]);  // parent, token
         if (d < Lout) dst[d] = rec.y;
@@ -827,24 +1082,42 @@ __global__ void __launch_bounds__(kMaxThreads) decode_kernel(DecodeParams p) {
 
 size_t decode_smem_bytes(int K, int V) { return make_layout(K, V).total; }
 
-int decode_block_threads(int K, int V) {
-  // about four candidates per thread when every token survives, at most 1024
-  long long want = ((long long)K * (V < 32 ? V : 32) + 3) / 4;
-  if (want < K) want = K;
-  int nt = (int)((want + 31) / 32 * 32);
-  if (nt < 64) nt = 64;
+int decode_block_threads(int K, int V, bool pruning) {
+  // one lane per beam entry for the stay candidates, about three extension candidates per
+  // ext lane, one chore warp.  With pruning on, a quarter of a large vocabulary (at least
+  // eight tokens) is assumed to survive a frame.
+  long long cols = V;
+  if (pruning) {
+    cols = V / 4;
+    if (cols < 8) cols = 8;
+    if (cols > V) cols = V;
+  }
+  const long long stay = ((long long)K + 31) / 32 * 32;
+  long long ext = ((long long)K * cols / 3 + 31) / 32 * 32;
+  if (ext < 32) ext = 32;
+  long long nt = stay + ext + 32;
   if (nt > kMaxThreads) nt = kMaxThreads;
-  return nt;
+  return (int)nt;
 }
 
 cudaError_t decode_prepare(int K, int V) {
-  return cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)decode_smem_bytes(K, V));
+  const int bytes = (int)decode_smem_bytes(K, V);
+  cudaError_t e = cudaFuncSetAttribute(decode_kernel<kSmallBlock>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(decode_kernel<kMaxThreads>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   if (p.B == 0) return cudaSuccess;
-  decode_kernel<<<p.B, decode_block_threads(p.K, p.V), decode_smem_bytes(p.K, p.V), s>>>(p);
+  int nt = p.block_threads > 0 ? p.block_threads : decode_block_threads(p.K, p.V, p.pruning != 0);
+  nt = (nt + 31) / 32 * 32;
+  if (nt < 96) nt = 96;  // a stay warp, an ext warp and the chore warp
+  if (nt > kMaxThreads) nt = kMaxThreads;
+  const size_t bytes = decode_smem_bytes(p.K, p.V);
+  if (nt <= kSmallBlock) decode_kernel<kSmallBlock><<<p.B, nt, bytes, s>>>(p);
+  else decode_kernel<kMaxThreads><<<p.B, nt, bytes, s>>>(p);
   return cudaGetLastError();
 }
 

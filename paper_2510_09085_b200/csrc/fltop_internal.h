@@ -12,33 +12,26 @@ struct __align__(8) Survivor {
   float logp;
 };
 
-// Prefix-trie node (one per distinct prefix of an utterance, 32 bytes).
-// Children of a node form a singly linked list (first_child / next_sibling);
-// child_filter has bit (token & 63) set for every child ever created, so that
-// "no such child yet" is decided without touching the list.
-struct __align__(32) TrieNode {
-  int32_t parent;        // node id of the prefix without its last token, -1 for the root
-  int32_t token;         // last token of the prefix, -1 for the root
-  int32_t first_child;   // head of the child list, -1 if none
-  int32_t next_sibling;  // next child of `parent`, -1 at the end
-  int32_t depth;         // number of tokens
-  int32_t pad;
-  unsigned long long child_filter;
+// Prefix-trie node: a back-pointer record, written once when a prefix enters
+// the beam and read only when hypotheses are written out.
+struct __align__(8) TrieNode {
+  int32_t parent;  // node id of the prefix without its last token, -1 for the root
+  int32_t token;   // last token of the prefix, -1 for the root
 };
 
 // Per-stream state header kept in HBM between stream_step calls.
 struct StateHeader {
   int32_t nbeam;      // live beam entries
-  int32_t n_nodes;    // trie nodes allocated (node 0 = empty prefix)
+  int32_t n_nodes;    // trie node ids handed out (node 0 = empty prefix)
   int32_t frames;     // frames consumed since the last reset
   int32_t status;     // sticky FLTOP_ST_* bits
   double offset;      // log-probability of the renormalisation point (see decode kernel)
   int32_t pad[2];
 };
 constexpr int kStateHeaderWords = sizeof(StateHeader) / 4;
-// beam arrays stored after the header, each K words (child_filter: 2K words):
-// node, last, par, parnode, pb, pnb, first, len, child_filter (2 words), tot
-constexpr int kStateWordsPerSlot = 11;
+// beam arrays stored after the header, each K words (fingerprints: 2K words each):
+// node, last, len, pb, pnb, tot, fingerprint, parent fingerprint
+constexpr int kStateWordsPerSlot = 10;
 inline size_t state_words(int K) { return kStateHeaderWords + (size_t)kStateWordsPerSlot * K; }
 
 struct PruneParams {
@@ -57,6 +50,8 @@ struct DecodeParams {
   int32_t B, T, V, K, blank, L;
   int32_t streaming;        // 0: reset at entry, no state kept.  1: state loaded / stored
   int32_t emit_default;     // streaming with flags == null: emit results?
+  int32_t block_threads;    // 0 = choose from K, V and whether pruning is on
+  int32_t pruning;          // 1 when R > 0 (fewer survivors than V expected)
   const int32_t* counts;    // [B*T] survivors per frame
   const Survivor* entries;  // [B*T*V]
   TrieNode* nodes;          // [B * nodes_per_utt]
@@ -71,7 +66,7 @@ struct DecodeParams {
 };
 
 size_t decode_smem_bytes(int K, int V);
-int decode_block_threads(int K, int V);
+int decode_block_threads(int K, int V, bool pruning);
 cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s);
 cudaError_t decode_prepare(int K, int V);  // one-time kernel attribute set-up

@@ -68,7 +68,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   if (!d_lengths || !d_tokens || !d_lens || !d_scores || !d_nhyp) return FLTOP_ERR_INVALID_ARG;
   if (T > 0 && (!d_logp || stride_t < vocab_size || stride_b < 0)) return FLTOP_ERR_INVALID_ARG;
   // the fixed scratch bounds the problem size
-  const int64_t nodes_per_utt = (int64_t)beam_width * (T > 0 ? T : 1) + 1;
+  const int64_t nodes_per_utt = (int64_t)((beam_width + 1) & ~1) * (T > 0 ? T : 1) + 2;
   if (vocab_size > kStaticMaxVocab || (int64_t)B * T > kStaticMaxFrames ||
       (int64_t)B * nodes_per_utt > kStaticMaxNodes)
     return FLTOP_ERR_CAPACITY;
@@ -94,7 +94,8 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   DecodeParams dp;
   dp.lengths = d_lengths; dp.flags = nullptr; dp.B = B; dp.T = T; dp.V = vocab_size;
   dp.K = beam_width; dp.blank = blank_id; dp.L = max_out_len; dp.streaming = 0;
-  dp.emit_default = 1; dp.counts = pp.counts; dp.entries = pp.entries;
+  dp.emit_default = 1; dp.block_threads = 0; dp.pruning = threshold_r > 0.f ? 1 : 0;
+  dp.counts = pp.counts; dp.entries = pp.entries;
   dp.nodes = reinterpret_cast<TrieNode*>(scratch + kCountsBytes + kEntriesBytes);
   dp.nodes_per_utt = nodes_per_utt; dp.state = nullptr;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
