@@ -66,10 +66,11 @@ namespace {
 constexpr int kMaxThreads = 1024;
 constexpr int kSmallBlock = 256;   // up to here every warp scans the histogram itself
 constexpr int kCache = 4;          // extension keys cached in registers per ext lane
-static_assert(kCache == 4, "the cached-key selects in P3 are written out for four keys");
+static_assert(kCache == 4, "the cached-score selects in P3 are written out for four scores");
 constexpr int kFastBins = 256;     // score histogram of the fast select
 constexpr float kBinsPerNat = 4.f;
 constexpr int kBinsPerLane = kFastBins / 32;
+static_assert(kBinsPerLane == 8, "a lane reads its eight bins with two 128-bit loads");
 constexpr int kListCap = 64;       // candidates of the cut bin ranked pairwise
 constexpr int kRadixBits = 8;      // exact fallback select
 constexpr int kBins = 1 << kRadixBits;
@@ -109,11 +110,6 @@ __device__ __forceinline__ float key_score(unsigned k) {
 __device__ __forceinline__ int score_bin(float s) {
   const int b = __float2int_rz(-s * kBinsPerNat);
   return min(kFastBins - 1, max(0, b));
-}
-// Bins are stored transposed so that the lane that owns bins
-// [8 l, 8 l + 8) reads them without bank conflicts.
-__device__ __forceinline__ int bin_addr(int bin) {
-  return ((bin & (kBinsPerLane - 1)) << 5) | (bin / kBinsPerLane);
 }
 
 // Fingerprint of a prefix extended by one token.
@@ -193,10 +189,10 @@ enum {
   SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_NBEAM_NEXT, SC_COUNT
 };
 
-// Slots of the beam's fingerprint table: a power of two, at least four times the beam width
-// (twice above 1024) so that probe sequences stay short.
+// Slots of the beam's fingerprint table: a power of two, sixteen times the beam width for
+// small beams (probe sequences of length one, almost always) and at least twice for large.
 __host__ __device__ inline int table_size(int K) {
-  const int want = K > 1024 ? 2 * K : 4 * K;
+  const int want = K <= 128 ? 16 * K : (K <= 1024 ? 4 * K : 2 * K);
   int n = 256;
   while (n < want) n <<= 1;
   return n;
@@ -289,48 +285,44 @@ struct Cut {
 // One warp turns the score histogram into the cut (all lanes get the result).
 __device__ __forceinline__ Cut scan_score_histogram(const unsigned* hist, int K) {
   const int lane = threadIdx.x & 31;
-  unsigned cnt[kBinsPerLane];
-  unsigned c = 0;
-#pragma unroll
-  for (int i = 0; i < kBinsPerLane; ++i) {
-    cnt[i] = hist[(i << 5) | lane];
-    c += cnt[i];
-  }
-  unsigned inc = c;
+  // lane l owns bins [8 l, 8 l + 8): inclusive prefix counts inside the lane, then over lanes
+  const uint4 lo4 = reinterpret_cast<const uint4*>(hist)[2 * lane];
+  const uint4 hi4 = reinterpret_cast<const uint4*>(hist)[2 * lane + 1];
+  int pre[kBinsPerLane];
+  pre[0] = (int)lo4.x; pre[1] = pre[0] + (int)lo4.y; pre[2] = pre[1] + (int)lo4.z;
+  pre[3] = pre[2] + (int)lo4.w; pre[4] = pre[3] + (int)hi4.x; pre[5] = pre[4] + (int)hi4.y;
+  pre[6] = pre[5] + (int)hi4.z; pre[7] = pre[6] + (int)hi4.w;
+  const int c = pre[7];
+  int inc = c;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const unsigned up = __shfl_up_sync(kFull, inc, o);
+    const int up = __shfl_up_sync(kFull, inc, o);
     if (lane >= o) inc += up;
   }
+  const int before = inc - c;
   Cut r;
-  const unsigned any = __ballot_sync(kFull, c != 0u);
+  const unsigned any = __ballot_sync(kFull, c != 0);
   r.first = any ? __ffs(any) - 1 : 0;
-  r.total = (int)__shfl_sync(kFull, inc, 31);
+  r.total = __shfl_sync(kFull, inc, 31);
   if (r.total <= K) {
     r.thr = kFastBins; r.left = 0; r.cut_count = 0; r.cut_base = r.total;
     return r;
   }
-  const unsigned hit = __ballot_sync(kFull, (int)inc >= K);
-  const int owner = __ffs(hit) - 1;
-  unsigned acc = inc - c;
-  int cut = 0;
-  unsigned cut_cnt = 0;
-  bool found = false;
+  // The inclusive prefix counts grow with the bin, so the cut bin is the number of bins
+  // whose count stays below K, the candidates above it are the largest such count, and the
+  // bin's own population follows from the smallest count that reaches K.
+  int n_below = 0, best_below = 0, first_reach = 0x7fffffff;
 #pragma unroll
   for (int i = 0; i < kBinsPerLane; ++i) {
-    if (!found) {
-      if ((int)(acc + cnt[i]) >= K) {
-        found = true;
-        cut = i;
-        cut_cnt = cnt[i];
-      } else {
-        acc += cnt[i];
-      }
-    }
+    const int v = before + pre[i];
+    const bool below = v < K;
+    n_below += below ? 1 : 0;
+    best_below = below ? max(best_below, v) : best_below;
+    first_reach = below ? first_reach : min(first_reach, v);
   }
-  r.thr = kBinsPerLane * owner + __shfl_sync(kFull, cut, owner);
-  r.cut_base = (int)__shfl_sync(kFull, acc, owner);
-  r.cut_count = (int)__shfl_sync(kFull, cut_cnt, owner);
+  r.thr = __reduce_add_sync(kFull, n_below);
+  r.cut_base = __reduce_max_sync(kFull, best_below);
+  r.cut_count = __reduce_min_sync(kFull, first_reach) - r.cut_base;
   r.left = K - r.cut_base;
   return r;
 }
@@ -387,15 +379,20 @@ __device__ __forceinline__ void divmod_small(int e, int d, float inv_d, int& q, 
   else if (r >= d) { ++q; r -= d; }
 }
 
-template <int MAXT>
+// KMAX / VMAX > 0: the shared-memory arrays are laid out for that beam width and vocabulary
+// whatever K and V are (K <= KMAX, V <= VMAX), so every array offset is a compile-time
+// constant; 0: laid out for the K and V of the call.
+template <int MAXT, int KMAX, int VMAX>
 __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
   const int K = p.K, V = p.V, blank = p.blank;
-  const Lay L = make_layout(K, V);
-  const int TS = table_size(K);
-  const int DW = dup_words(K, V);
-  const int NSL = node_stage_len(K);
+  const int KS = KMAX > 0 ? KMAX : K;  // strides of the per-entry / per-token arrays
+  const int VS = VMAX > 0 ? VMAX : V;
+  const Lay L = make_layout(KS, VS);
+  const int TS = table_size(KS);
+  const int DW = dup_words(KS, VS);
+  const int NSL = node_stage_len(KS);
   const unsigned tmask = (unsigned)TS - 1u;
   const unsigned lt_mask = (1u << lane) - 1u;
 
@@ -407,7 +404,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   unsigned long long* const warp_sums = reinterpret_cast<unsigned long long*>(smem + L.warp_sums);
   float* const st_pb = reinterpret_cast<float*>(smem + L.st_pb);
   float* const st_pnb = reinterpret_cast<float*>(smem + L.st_pnb);
-  unsigned* const st_key = reinterpret_cast<unsigned*>(smem + L.st_key);
+  float* const st_tot = reinterpret_cast<float*>(smem + L.st_key);  // lse(st_pb, st_pnb)
   unsigned* const dup_base = reinterpret_cast<unsigned*>(smem + L.dup);
   TrieNode* const nstage = reinterpret_cast<TrieNode*>(smem + L.nstage);
   int* const jpos_base = reinterpret_cast<int*>(smem + L.jpos);
@@ -454,7 +451,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   // ---- initialise shared state -------------------------------------------------
   for (int i = tid; i < 2 * DW; i += NT) dup_base[i] = 0u;
   for (int i = tid; i < 2 * TS; i += NT) tab_base[i] = kEmptySlot;
-  for (int i = tid; i < 2 * V; i += NT) lpv_base[i] = neg_inf();
+  for (int i = tid; i < 2 * VS; i += NT) lpv_base[i] = neg_inf();
   for (int i = tid; i < 2 * kFastBins; i += NT) hist_base[i] = 0u;
   if (tid < SC_COUNT) scal[tid] = 0;
   int created = 0, live_sum = 0;
@@ -518,8 +515,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
 
   const int32_t* counts = p.counts + (int64_t)b * p.T;
   const Survivor* entries = p.entries + (int64_t)b * p.T * V;
-  auto svbuf = [&](int t) -> Survivor* { return sv_base + (t & 3) * V; };
-  auto lpvbuf = [&](int t) -> float* { return lpv_base + (t & 1) * V; };
+  auto svbuf = [&](int t) -> Survivor* { return sv_base + (t & 3) * VS; };
+  auto lpvbuf = [&](int t) -> float* { return lpv_base + (t & 1) * VS; };
 
   // Chore warp: the log-probability table and the constants of frame t1 (its survivors are
   // in shared memory), and the table of frame t1 - 1 forgotten (t1 > 0).
@@ -550,7 +547,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         bl = __shfl_sync(kFull, lp, src);
       }
     }
-    int* jp_new = jpos_base + (t1 & 1) * V;
+    int* jp_new = jpos_base + (t1 & 1) * VS;
     for (int j = lane; j < S1; j += 32) jp_new[sn[j].token] = j - ((bj >= 0 && j > bj) ? 1 : 0);
     if (lane == 0) {
       FrameInfo f;
@@ -586,15 +583,15 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     const int par = t & 1, nxt = cur ^ 1;
     const Survivor* const sv = svbuf(t);
     const float* const lpv = lpvbuf(t);
-    const Hot* const hc = hot_base + cur * K;
-    Hot* const hn = hot_base + nxt * K;
-    const Ident* const id_c = ident_base + cur * K;
-    Ident* const id_n = ident_base + nxt * K;
-    const Where* const wh_c = where_base + cur * K;
-    Where* const wh_n = where_base + nxt * K;
+    const Hot* const hc = hot_base + cur * KS;
+    Hot* const hn = hot_base + nxt * KS;
+    const Ident* const id_c = ident_base + cur * KS;
+    Ident* const id_n = ident_base + nxt * KS;
+    const Where* const wh_c = where_base + cur * KS;
+    Where* const wh_n = where_base + nxt * KS;
     unsigned* const hist = hist_base + par * kFastBins;
     unsigned* const dupbits = dup_base + par * DW;
-    const int* const jpos = jpos_base + par * V;
+    const int* const jpos = jpos_base + par * VS;
     const unsigned* const tab_c = tab_base + par * TS;
     unsigned* const tab_n = tab_base + (par ^ 1) * TS;
     int* const sc_c = scal + par * SC_PER_FRAME;
@@ -616,9 +613,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     auto ext_token = [&](int j) -> int { return sv[sv_index(j)].token; };
     // extension candidate e = q * Snb + j names a prefix that is already in the beam
     auto merged = [&](int e) -> bool { return (dupbits[e >> 5] >> (e & 31)) & 1u; };
-    auto count = [&](float score) { atomicAdd(&hist[bin_addr(score_bin(score))], 1u); };
+    auto count = [&](float score) { atomicAdd(&hist[score_bin(score)], 1u); };
     // stay candidate of entry q, including the prefix merge
-    auto stay_eval = [&](int q) -> unsigned {
+    auto stay_eval = [&](int q) -> float {
       const Hot e = hc[q];
       const float npb = e.tot + fi.lp_blank;
       float npnb = neg_inf();
@@ -631,7 +628,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           const float dup = ((pe.last == e.last) ? pe.pb : pe.tot) + le;
           if (dup != neg_inf()) {  // the parent's extension by last(q) names this prefix
             npnb = lse2(npnb, dup);
-            atomicSub(&hist[bin_addr(score_bin(dup))], 1u);
+            atomicSub(&hist[score_bin(dup)], 1u);
             const int ed = pq * Snb + jpos[e.last];
             atomicOr(&dupbits[ed >> 5], 1u << (ed & 31));
           }
@@ -640,10 +637,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       st_pb[q] = npb;
       st_pnb[q] = npnb;
       const float tot = lse2(npb, npnb);
-      const unsigned key = score_key(tot);
-      st_key[q] = key;
-      if (key) count(tot);
-      return key;
+      st_tot[q] = tot;
+      if (tot != neg_inf()) count(tot);
+      return tot;
     };
     // this lane's extension candidates: e_first, e_first + NX, ... as (q, j) pairs
     int q0 = 0, j0 = 0;
@@ -660,13 +656,11 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     };
 
     // ---- P1: every candidate is evaluated once and counted -----------------------------
-    unsigned kc[kCache];
-    unsigned kstay = 0u;
+    float kc[kCache];  // this ext lane's first extension scores (-inf: none)
 #pragma unroll
-    for (int k = 0; k < kCache; ++k) kc[k] = 0u;
+    for (int k = 0; k < kCache; ++k) kc[k] = neg_inf();
     if (is_stay) {
-      if (tid < nb) kstay = stay_eval(tid);
-      for (int i = tid + NS; i < nb; i += NS) stay_eval(i);
+      for (int i = tid; i < nb; i += NS) stay_eval(i);
     } else if (is_ext) {
       divmod_small(xl, Sdiv, fi.inv_s, q0, j0);
       int q = q0, j = j0;
@@ -675,7 +669,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         if (xl + k * NX < next) {
           const float sc = ext_score(hc[q], j);
           step(q, j);
-          kc[k] = score_key(sc);
+          kc[k] = sc;
           if (sc != neg_inf()) count(sc);
         }
       }
@@ -764,7 +758,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     int nbn = min(cut.total, K);
     TrieNode* const nst = nstage + par * NSL;
     // the frame's nodes get ids n_nodes .. n_nodes + nbn - 1 (the slots of stays stay unused)
-    const bool arena_ok = (int64_t)n_nodes + NSL <= p.nodes_per_utt;
+    const bool arena_ok = (int64_t)n_nodes + ((K + 1) & ~1) <= p.nodes_per_utt;
 
     // ---- P3: selected candidates take their slots in the next beam ---------------------
     auto place_stay = [&](int q, unsigned key, int slot) {
@@ -805,13 +799,13 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     };
 
     if (take_all || use_list) {
-      // key thresholds of the cut: key > k_hi is above the cut bin, key > k_lo is in it or above
-      const unsigned k_lo = (cut.thr >= kFastBins - 1)
-                                ? 0u
-                                : score_key(-(float)(cut.thr + 1) * (1.f / kBinsPerNat));
-      const unsigned k_hi = take_all ? k_lo
-                                     : (cut.thr == 0 ? 0xffffffffu
-                                                     : score_key(-(float)cut.thr * (1.f / kBinsPerNat)));
+      // the cut as scores (bin edges): score > f_hi is above the cut bin, score > f_lo is in
+      // it or above.  A score of -inf passes neither.
+      const float f_lo = (cut.thr >= kFastBins - 1) ? neg_inf()
+                                                    : -(float)(cut.thr + 1) * (1.f / kBinsPerNat);
+      const float f_hi = take_all ? f_lo
+                                  : (cut.thr == 0 ? __int_as_float(0x7f800000)
+                                                  : -(float)cut.thr * (1.f / kBinsPerNat));
       // P3a: every candidate above the cut bin takes a beam slot and is noted there; stays
       // fill the beam from slot 0 upwards, extensions from the last slot downwards.
       auto list_add = [&](unsigned key, int id) {
@@ -822,79 +816,68 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         }
       };
       if (is_stay) {
-        for (int base = 0; base < nb || base == 0; base += NS) {
+        // stays are dense: one ballot per round, the warp's places taken by its first lane
+        for (int base = 0; base < nb; base += NS) {
           const int i = base + tid;
-          const unsigned key = base == 0 ? kstay : (i < nb ? st_key[i] : 0u);
-          const bool sel = key > k_hi;
+          const float sc = i < nb ? st_tot[i] : neg_inf();
+          const bool sel = sc > f_hi;
           const unsigned m = __ballot_sync(kFull, sel);
           if (m) {
             int at = 0;
             if (lane == 0) at = atomicAdd(&sc_c[SC_SLOT], __popc(m));
             at = __shfl_sync(kFull, at, 0) + __popc(m & lt_mask);
             if (sel && at < K) {
-              sel_key[at] = key;
+              sel_key[at] = score_key(sc);
               sel_id[at] = i << 16;
             }
           }
-          if (!sel && key > k_lo) list_add(key, i << 16);
+          if (!sel && sc > f_lo) list_add(score_key(sc), i << 16);
         }
       } else if (is_ext) {
-        // `n` consecutive places for this lane, n <= 7 (warp-collective)
-        auto claim = [&](int n) -> int {
-          const unsigned b0 = __ballot_sync(kFull, n & 1);
-          const unsigned b1 = __ballot_sync(kFull, n & 2);
-          const unsigned b2 = __ballot_sync(kFull, n & 4);
-          if (!(b0 | b1 | b2)) return 0;
+        // extensions in the cut bin or above: the lanes of a warp that arrive here together
+        // take their places with one atomic
+        auto settle = [&](int e, int q, int j, float sc) {
+          if (merged(e)) return;
+          const unsigned key = score_key(sc);
+          const int id = (q << 16) | (j + 1);
+          const bool sure = sc > f_hi;
+          const unsigned act = __activemask();
+          const unsigned ms = __ballot_sync(act, sure);
+          const unsigned mine = sure ? ms : (act & ~ms);
+          int* const counter = sure ? &sc_c[SC_SLOT_E] : &sc_c[SC_LISTN];
+          const int leader = __ffs(mine) - 1;
           int at = 0;
-          if (lane == 0)
-            at = atomicAdd(&sc_c[SC_SLOT_E], __popc(b0) + 2 * __popc(b1) + 4 * __popc(b2));
-          at = __shfl_sync(kFull, at, 0);
-          return at + __popc(b0 & lt_mask) + 2 * __popc(b1 & lt_mask) + 4 * __popc(b2 & lt_mask);
-        };
-        auto note = [&](int at, unsigned key, int id) {
-          const int slot = nbn - 1 - at;
-          if ((unsigned)slot < (unsigned)K) {
-            sel_key[slot] = key;
-            sel_id[slot] = id;
+          if (lane == leader) at = atomicAdd(counter, __popc(mine));
+          at = __shfl_sync(mine, at, leader) + __popc(mine & lt_mask);
+          if (sure) {
+            const int slot = nbn - 1 - at;
+            if ((unsigned)slot < (unsigned)K) {
+              sel_key[slot] = key;
+              sel_id[slot] = id;
+            }
+          } else if (at < kListCap) {
+            list_key[at] = key;
+            list_id[at] = id;
           }
         };
-        // cached candidates: settle which are selected, then take the places in one go
         unsigned want = 0u;  // bit k: cached candidate k is in the cut bin or above
 #pragma unroll
-        for (int k = 0; k < kCache; ++k) want |= (kc[k] > k_lo ? 1u : 0u) << k;
-        unsigned selm = 0u;
-        int ids[kCache];
-#pragma unroll
-        for (int k = 0; k < kCache; ++k) ids[k] = 0;
+        for (int k = 0; k < kCache; ++k) want |= (kc[k] > f_lo ? 1u : 0u) << k;
         for (unsigned m = want; m; m &= m - 1) {
           const int k = __ffs(m) - 1;
-          if (merged(xl + k * NX)) continue;
-          const unsigned key = k == 0 ? kc[0] : k == 1 ? kc[1] : k == 2 ? kc[2] : kc[3];
           int q, j;
           nth(k, q, j);
-          const int id = (q << 16) | (j + 1);
-          if (key > k_hi) {
-            selm |= 1u << k;
-            if (k == 0) ids[0] = id; else if (k == 1) ids[1] = id; else if (k == 2) ids[2] = id; else ids[3] = id;
-          } else {
-            list_add(key, id);
-          }
+          settle(xl + k * NX, q, j, k == 0 ? kc[0] : k == 1 ? kc[1] : k == 2 ? kc[2] : kc[3]);
         }
-        int at = claim(__popc(selm));
-#pragma unroll
-        for (int k = 0; k < kCache; ++k)
-          if ((selm >> k) & 1u) note(at++, kc[k], ids[k]);
         // candidates beyond the cache are evaluated again
-        int q, j;
-        nth(kCache, q, j);
-        for (int base = kCache * NX; base < next; base += NX) {
-          unsigned key = (xl + base < next) ? ext_key(hc[q], j) : 0u;
-          if (key > k_lo && merged(xl + base)) key = 0u;
-          const bool sel = key > k_hi;
-          const int a1 = claim(sel ? 1 : 0);
-          if (sel) note(a1, key, (q << 16) | (j + 1));
-          else if (key > k_lo) list_add(key, (q << 16) | (j + 1));
-          step(q, j);
+        if (kCache * NX < next) {
+          int q, j;
+          nth(kCache, q, j);
+          for (int e = xl + kCache * NX; e < next; e += NX) {
+            const float sc = ext_score(hc[q], j);
+            if (sc > f_lo) settle(e, q, j, sc);
+            step(q, j);
+          }
         }
       }
       __syncthreads();  // B3: every selected candidate is noted, the cut bin's members listed
@@ -926,7 +909,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       // ---- exact fallback: radix select over the integer keys ------------------------
       auto for_each_candidate = [&](auto&& f) {
         if (is_stay) {
-          for (int i = tid; i < nb; i += NS) f(st_key[i], i << 16);
+          for (int i = tid; i < nb; i += NS) f(score_key(st_tot[i]), i << 16);
         } else if (is_ext) {
           int q = q0, j = j0;
           for (int e = xl; e < next; e += NX) {
@@ -1016,9 +999,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     }
   }
 
-  const Hot* const hc = hot_base + cur * K;
-  const Ident* const id_c = ident_base + cur * K;
-  const Where* const wh_c = where_base + cur * K;
+  const Hot* const hc = hot_base + cur * KS;
+  const Ident* const id_c = ident_base + cur * KS;
+  const Where* const wh_c = where_base + cur * KS;
 
   // ---- keep the beam for the next chunk (streaming) -----------------------------------
   if (p.streaming) {
@@ -1080,7 +1063,22 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
 
 }  // namespace
 
-size_t decode_smem_bytes(int K, int V) { return make_layout(K, V).total; }
+// Layout variants: small beams over a character or a subword vocabulary get compile-time
+// array offsets, everything else the generic kernel.
+enum Variant { kCharBeam64, kSubwordBeam64, kGeneric };
+Variant pick_variant(int K, int V) {
+  if (K <= 64 && V <= 32) return kCharBeam64;
+  if (K <= 64 && V <= 1024) return kSubwordBeam64;
+  return kGeneric;
+}
+
+size_t decode_smem_bytes(int K, int V) {
+  switch (pick_variant(K, V)) {
+    case kCharBeam64: return make_layout(64, 32).total;
+    case kSubwordBeam64: return make_layout(64, 1024).total;
+    default: return make_layout(K, V).total;
+  }
+}
 
 int decode_block_threads(int K, int V, bool pruning) {
   // one lane per beam entry for the stay candidates, about three extension candidates per
@@ -1100,13 +1098,29 @@ int decode_block_threads(int K, int V, bool pruning) {
   return (int)nt;
 }
 
-cudaError_t decode_prepare(int K, int V) {
-  const int bytes = (int)decode_smem_bytes(K, V);
-  cudaError_t e = cudaFuncSetAttribute(decode_kernel<kSmallBlock>,
+namespace {
+template <int KMAX, int VMAX>
+cudaError_t prepare_variant(int bytes) {
+  cudaError_t e = cudaFuncSetAttribute(decode_kernel<kSmallBlock, KMAX, VMAX>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(decode_kernel<kMaxThreads>,
+  return cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX>,
                               cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+template <int KMAX, int VMAX>
+void launch_variant(const DecodeParams& p, int nt, size_t bytes, cudaStream_t s) {
+  if (nt <= kSmallBlock) decode_kernel<kSmallBlock, KMAX, VMAX><<<p.B, nt, bytes, s>>>(p);
+  else decode_kernel<kMaxThreads, KMAX, VMAX><<<p.B, nt, bytes, s>>>(p);
+}
+}  // namespace
+
+cudaError_t decode_prepare(int K, int V) {
+  const int bytes = (int)decode_smem_bytes(K, V);
+  switch (pick_variant(K, V)) {
+    case kCharBeam64: return prepare_variant<64, 32>(bytes);
+    case kSubwordBeam64: return prepare_variant<64, 1024>(bytes);
+    default: return prepare_variant<0, 0>(bytes);
+  }
 }
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
@@ -1116,8 +1130,11 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   if (nt < 96) nt = 96;  // a stay warp, an ext warp and the chore warp
   if (nt > kMaxThreads) nt = kMaxThreads;
   const size_t bytes = decode_smem_bytes(p.K, p.V);
-  if (nt <= kSmallBlock) decode_kernel<kSmallBlock><<<p.B, nt, bytes, s>>>(p);
-  else decode_kernel<kMaxThreads><<<p.B, nt, bytes, s>>>(p);
+  switch (pick_variant(p.K, p.V)) {
+    case kCharBeam64: launch_variant<64, 32>(p, nt, bytes, s); break;
+    case kSubwordBeam64: launch_variant<64, 1024>(p, nt, bytes, s); break;
+    default: launch_variant<0, 0>(p, nt, bytes, s); break;
+  }
   return cudaGetLastError();
 }
 
