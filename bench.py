@@ -1,6 +1,7 @@
 """Benchmark of the frame-pruned CTC prefix beam search library.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --report FILE     # all five workloads, written as a markdown table
 
 One step = one pass of the whole hot path (prune, extend, merge, select, trie
 append, readback) over one synthetic wav2vec2-shaped batch: B=64 utterances,
@@ -316,6 +317,149 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def _time_decode(dec, x, ln, flush, reps=7, warm=2):
+    """Best-of device times (ms) of the whole call and of its prune and decode kernels."""
+    import torch
+    best = None
+    for i in range(warm + reps):
+        flush.fill_(i & 0xff)
+        t0, t1 = torch.cuda.Event(True), torch.cuda.Event(True)
+        t0.record()
+        dec.decode(x, ln)
+        t1.record()
+        t1.synchronize()
+        if i >= warm:
+            pk, dk = dec.last_kernel_ms()
+            cur = (t0.elapsed_time(t1), pk, dk)
+            best = cur if best is None or cur[0] < best[0] else best
+    return best
+
+
+def _oracle_top1(wl, K, r, threads):
+    """Top-1 sequence of every utterance from the CPU oracle (utterances in parallel threads)."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+
+    def one(b):
+        res = oracle.decode(wl.emissions[b:b + 1], wl.lengths[b:b + 1], wl.blank_id, K, r)
+        return res.hyps(0)[0][0]
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(one, range(len(wl.lengths))))
+
+
+def run_report(args):
+    """All five workloads on one GPU; a markdown table goes to args.report."""
+    import torch
+    from paper_2510_09085_b200 import binding, workloads
+    peak, peak_kind = _peaks()
+    cores = len(os.sched_getaffinity(0))
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    rows = []
+
+    def measure(wl, K, r, label, top1_ref=None):
+        B, T, V = wl.emissions.shape
+        x = torch.from_numpy(wl.emissions).cuda()
+        ln = torch.from_numpy(wl.lengths).cuda()
+        dec = binding.Decoder(V, wl.blank_id, K, r, B, T)
+        dec.set_profiling(True)
+        ms, pk, dk = _time_decode(dec, x, ln, flush)
+        st = dec.last_call_stats()
+        assert int((dec.status != 0).sum()) == 0
+        frames = int(wl.lengths.sum())
+        pbytes = st["frames"] * (4 * V + 4) + st["survivors"] * SURVIVOR_BYTES
+        dbytes = (st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES
+                  + NODE_BYTES * (st["live_hypotheses_sum"] + st["frames"])
+                  + 4 * int(dec.lens.sum()) + 8 * int(dec.nhyp.sum()) + 8 * B)
+        agree = None
+        if top1_ref is not None:
+            agree = sum(dec.hyps(b)[0][0] == top1_ref[b] for b in range(B)) / B
+        row = {"workload": label, "K": K, "r": r, "frames_per_s": frames / (ms * 1e-3),
+               "utt_per_s": B / (ms * 1e-3), "ms": ms, "prune_ms": pk, "decode_ms": dk,
+               "hbm_frac_step": (pbytes + dbytes) / (ms * 1e-3) / 1e9 / peak,
+               "prune_gbs": pbytes / (pk * 1e-3) / 1e9 if pk > 0 else 0.0,
+               "ns_per_frame_step": 1e6 * dk / max(1, int(wl.lengths.max())),
+               "beam_state_bytes": dec.beam_state_bytes,
+               "mean_survivors": st["survivors"] / max(1, st["frames"]),
+               "mean_live": st["live_hypotheses_sum"] / max(1, st["frames"]), "top1_agree": agree}
+        rows.append(row)
+        dec.close()
+        print(json.dumps(row), file=sys.stderr, flush=True)
+        return row
+
+    pr1 = workloads.workload_pr1()
+    for r in pr1.thresholds:
+        measure(pr1, pr1.beam_width, r, "0 pr1")
+    wav = workloads.workload_wav2vec2()
+    for r in wav.thresholds:
+        measure(wav, wav.beam_width, r, "1 wav2vec2")
+    for K in workloads.SWEEP_BEAMS:
+        t0 = time.perf_counter()
+        ref = None if args.skip_oracle else _oracle_top1(wav, K, 0.0, cores)
+        print(f"oracle r=0 K={K}: {time.perf_counter() - t0:.1f} s on {cores} threads",
+              file=sys.stderr, flush=True)
+        for r in workloads.SWEEP_THRESHOLDS:
+            measure(wav, K, r, "2 sweep", ref)
+    sub = workloads.workload_subword()
+    for r in sub.thresholds:
+        measure(sub, sub.beam_width, r, "3 subword")
+    # streaming: 1024 streams, 16-frame chunks, beam state carried in the handle
+    stw = workloads.workload_streaming()
+    S, T, V = stw.emissions.shape
+    C, K, r = stw.chunk_frames, stw.beam_width, stw.thresholds[0]
+    x = torch.from_numpy(stw.emissions).cuda()
+    dec = binding.Decoder(V, 0, K, r, S, T, max_chunk_frames=C)
+    full = torch.full((S,), C, dtype=torch.int32, device="cuda")
+    n = T // C
+    chunks = [x[:, i * C:(i + 1) * C].contiguous() for i in range(n)]
+    first = torch.full((S,), 1, dtype=torch.uint8, device="cuda")
+    mid = torch.zeros((S,), dtype=torch.uint8, device="cuda")
+    last = torch.full((S,), 2, dtype=torch.uint8, device="cuda")
+    lat, total = [], None
+    for rep in range(3):
+        torch.cuda.synchronize()
+        t_all = time.perf_counter()
+        for i in range(n):
+            flags = first if i == 0 else (last if i == n - 1 else mid)
+            t0 = time.perf_counter()
+            dec.stream_step(chunks[i], full, flags, readback=(i == n - 1))
+            torch.cuda.synchronize()
+            if rep > 0:
+                lat.append(time.perf_counter() - t0)
+        dt = time.perf_counter() - t_all
+        total = dt if total is None or dt < total else total
+    assert int((dec.status != 0).sum()) == 0
+    lat = np.array(lat) * 1e3
+    stream_row = {"workload": "4 streaming", "K": K, "r": r, "frames_per_s": S * T / total,
+                  "p50_ms": float(np.percentile(lat, 50)), "p99_ms": float(np.percentile(lat, 99)),
+                  "beam_state_bytes": dec.beam_state_bytes}
+    print(json.dumps(stream_row), file=sys.stderr, flush=True)
+    dec.close()
+    # CPU oracle, single thread, on a sample of the wav2vec2 workload (a reported baseline)
+    order = np.argsort(wav.lengths)
+    sample = [int(i) for i in order[::8]]
+    cpu_p, _ = _oracle_frames_per_s(wav, R_PRUNED, sample)
+    cpu_0, _ = _oracle_frames_per_s(wav, 0.0, sample)
+
+    with open(args.report, "w") as f:
+        f.write(f"Measured on one B200, HBM peak {peak:.0f} GB/s ({peak_kind}); host threads {cores}.\n\n")
+        f.write("| cfg | K | r | frames/s | utt/s | step ms | HBM frac (step) | prune GB/s | "
+                "ns / frame step | beam-state MB | mean survivors | mean live hyps | top-1 vs r=0 oracle |\n")
+        f.write("|---|---|---|---|---|---|---|---|---|---|---|---|---|\n")
+        for w in rows:
+            ag = "" if w["top1_agree"] is None else f"{100 * w['top1_agree']:.1f} %"
+            f.write(f"| {w['workload']} | {w['K']} | {w['r']:g} | {w['frames_per_s']:.3g} | "
+                    f"{w['utt_per_s']:.3g} | {w['ms']:.3f} | {100 * w['hbm_frac_step']:.3f} % | "
+                    f"{w['prune_gbs']:.0f} | {w['ns_per_frame_step']:.0f} | "
+                    f"{w['beam_state_bytes'] / 1e6:.1f} | {w['mean_survivors']:.2f} | "
+                    f"{w['mean_live']:.1f} | {ag} |\n")
+        f.write(f"\nStreaming (cfg 4, K={K}, r={r:g}, 1024 streams x 100 chunks of 16 frames): "
+                f"{stream_row['frames_per_s']:.3g} frames/s aggregate, chunk latency p50 "
+                f"{stream_row['p50_ms']:.3f} ms, p99 {stream_row['p99_ms']:.3f} ms (host wall clock, "
+                f"call to stream sync), beam state {stream_row['beam_state_bytes'] / 1e6:.1f} MB.\n")
+        f.write(f"\nCPU oracle, one thread, 8 of the 64 wav2vec2 utterances, K=50: "
+                f"{cpu_p:.0f} frames/s at r=1e-3, {cpu_0:.0f} frames/s at r=0.\n")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -323,8 +467,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--report", metavar="FILE", help="measure all five workloads, write a table")
+    ap.add_argument("--skip-oracle", action="store_true", help="--report without top-1 agreement")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.report:
+        run_report(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -242,3 +242,34 @@ def test_exact_ties_keep_a_valid_beam():
         assert sc <= full[seq] + TOL
     np.testing.assert_allclose(sorted(s for _, s in got), sorted(s for _, s in ref), atol=TOL)
     d.close()
+
+
+# ------------------------------------------------------------------ launch shape / large V
+def test_results_do_not_depend_on_the_block_size():
+    # threads per utterance block is a tuning knob: every setting must give the same beam
+    em, ln = W.make_small(31, 4, 40, 120, 32)
+    ref = None
+    for nt in (96, 128, 256, 512, 1024):
+        B, T, V = em.shape
+        d = _binding().Decoder(V, 0, 20, 1e-2, B, T)
+        d.set_block_threads(nt)
+        d.decode(_dev(em), _dev(ln))
+        torch.cuda.synchronize()
+        assert (d.status.cpu().numpy()[:B] == 0).all()
+        got = [d.hyps(b) for b in range(B)]
+        if ref is None:
+            ref = got
+        else:
+            assert got == ref, f"block of {nt} threads changed the result"
+        d.close()
+
+
+def test_large_vocabulary_prefixes_leave_and_reenter():
+    # vocabulary far above 64 tokens with a tiny beam on flat rows: prefixes are evicted and
+    # derived again all the time, and every re-entry must merge with its descendants in the beam
+    from tests.refs import py_decode
+    em, ln = W.make_small(77, 3, 30, 70, 300, hard_fraction=0.6, boost_easy=1.5)
+    revivals = sum(py_decode(em[b, : ln[b]], 0, 5, oracle.log_r(0.02)).revivals for b in range(3))
+    assert revivals > 0
+    compare_batch(em, ln, 0, 5, 0.02)
+    compare_batch(em, ln, 0, 3, 0.0)
