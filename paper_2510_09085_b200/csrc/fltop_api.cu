@@ -124,7 +124,7 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.lengths = d_lengths; dp.flags = d_flags; dp.B = B; dp.T = T; dp.V = h->cfg.vocab_size;
   dp.K = h->cfg.beam_width; dp.blank = h->cfg.blank_id; dp.L = h->cfg.max_out_len;
   dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
-  dp.block_threads = h->block_threads; dp.pruning = h->cfg.threshold_r > 0.f ? 1 : 0;
+  dp.block_threads = h->block_threads; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
   dp.counts = h->counts; dp.entries = h->entries; dp.nodes = h->nodes;
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;

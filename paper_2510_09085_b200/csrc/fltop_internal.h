@@ -51,7 +51,7 @@ struct DecodeParams {
   int32_t streaming;        // 0: reset at entry, no state kept.  1: state loaded / stored
   int32_t emit_default;     // streaming with flags == null: emit results?
   int32_t block_threads;    // 0 = choose from K, V and whether pruning is on
-  int32_t pruning;          // 1 when R > 0 (fewer survivors than V expected)
+  int32_t pruning;          // 1 when R is large enough that few tokens survive a frame
   const int32_t* counts;    // [B*T] survivors per frame
   const Survivor* entries;  // [B*T*V]
   TrieNode* nodes;          // [B * nodes_per_utt]
