@@ -139,7 +139,8 @@ int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t 
  * library image, FLTOP_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the
  * process exits.  Consequently:
  *   - the problem must fit: vocab_size <= FLTOP_STATIC_MAX_VOCAB, B*T <=
- *     FLTOP_STATIC_MAX_FRAMES, B*(beam_width*T + 1) <= FLTOP_STATIC_MAX_NODES; anything
+ *     FLTOP_STATIC_MAX_FRAMES, B*(K2*T + 2) <= FLTOP_STATIC_MAX_NODES with K2 = beam_width
+ *     rounded up to an even number; anything
  *     larger returns FLTOP_ERR_CAPACITY and launches nothing;
  *   - it runs on the CURRENT device.  The first call on each device looks up the array's
  *     device address (cudaGetSymbolAddress) before launching; make that first call outside
