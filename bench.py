@@ -32,6 +32,9 @@ UNIT = "frames/s"
 BATCH, BEAM, R_PRUNED = 64, 50, 1e-3
 L2_FLUSH_BYTES = 256 << 20
 NODE_BYTES, SURVIVOR_BYTES = 8, 8
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch on the default workload
+# (profiles/decode_kernel_wav2vec2_B64_K50_full.txt); None whenever the kernel has changed since
+DECODE_DRAM_BYTES = 9.31e6
 
 
 def _peaks():
@@ -295,7 +298,7 @@ def run_ours(args):
         "gpu_launches": launches,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved,
-                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": (DECODE_DRAM_BYTES if args.workload == "wav2vec2" and not args.batch else None),
                      "peak_source": f"{peak_kind} copy bandwidth",
                      "bytes_per_launch": db, "ms_per_launch": dk_ms,
                      "note": "latency-bound serial frame chain: max_frames dependent steps"},
