@@ -56,6 +56,16 @@ def _load():
                                            c.c_void_p]
         lib.oracle_stream_results.restype = c.c_int
         lib.oracle_stream_results.argtypes = [c.c_void_p] + [c.c_void_p] * 5 + [c.c_int]
+        lib.oracle_stream_options.restype = None
+        lib.oracle_stream_options.argtypes = [c.c_void_p, c.c_int, c.c_double]
+        lib.oracle_prune_topn.restype = None
+        lib.oracle_prune_topn.argtypes = [c.c_void_p, c.c_int64, c.c_int, c.c_float, c.c_int,
+                                          c.c_void_p, c.c_void_p]
+        lib.oracle_decode_opt.restype = None
+        lib.oracle_decode_opt.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_void_p, c.c_int,
+                                          c.c_int, c.c_int, c.c_int, c.c_int, c.c_float, c.c_int,
+                                          c.c_double, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p,
+                                          c.c_void_p, c.c_void_p, c.c_void_p]
         lib.oracle_decode.restype = None
         lib.oracle_decode.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_void_p, c.c_int,
                                       c.c_int, c.c_int, c.c_int, c.c_int, c.c_float, c.c_int,
@@ -73,14 +83,17 @@ def log_r(r: float) -> np.float32:
     return np.float32(_load().oracle_log_r(float(np.float32(r))))
 
 
-def prune(lp: np.ndarray, r: float):
-    """Survivor mask [.., V] (bool) and count [..] of every frame of ``lp`` [.., V]."""
+def prune(lp: np.ndarray, r: float, top_n: int = 0):
+    """Survivor mask [.., V] (bool) and count [..] of every frame of ``lp`` [.., V].
+
+    ``top_n`` > 0 keeps at most the top_n most probable tokens of a frame (N of Algorithm 1)."""
     lp = np.ascontiguousarray(lp, dtype=np.float32)
     V = lp.shape[-1]
     n = lp.size // V if V else 0
     keep = np.zeros(lp.shape, dtype=np.uint8)
     counts = np.zeros(lp.shape[:-1], dtype=np.int32)
-    _load().oracle_prune(_ptr(lp), n, V, float(np.float32(r)), _ptr(keep), _ptr(counts))
+    _load().oracle_prune_topn(_ptr(lp), n, V, float(np.float32(r)), int(top_n), _ptr(keep),
+                              _ptr(counts))
     return keep.astype(bool), counts
 
 
@@ -98,8 +111,10 @@ class DecodeResult:
 
 
 def decode(lp: np.ndarray, lengths, blank: int, K: int, r: float, max_len: int | None = None,
-           want_masks: bool = False) -> DecodeResult:
-    """Frame-pruned CTC prefix beam search of a padded batch ``lp`` [B,T,V]."""
+           want_masks: bool = False, top_n: int = 0, beam_threshold: float = 0.0) -> DecodeResult:
+    """Frame-pruned CTC prefix beam search of a padded batch ``lp`` [B,T,V].
+
+    ``top_n`` and ``beam_threshold`` are N and beam_threshold of Algorithm 1 (0 = off)."""
     lp = np.ascontiguousarray(lp, dtype=np.float32)
     B, T, V = lp.shape
     lengths = np.ascontiguousarray(lengths, dtype=np.int32)
@@ -110,9 +125,10 @@ def decode(lp: np.ndarray, lengths, blank: int, K: int, r: float, max_len: int |
     nhyp = np.zeros(B, dtype=np.int32)
     keep = np.zeros((B, T, V), dtype=np.uint8) if want_masks else None
     counts = np.zeros((B, T), dtype=np.int32) if want_masks else None
-    _load().oracle_decode(_ptr(lp), T * V, V, _ptr(lengths), B, T, V, blank, K,
-                          float(np.float32(r)), L, _ptr(tokens), _ptr(lens), _ptr(scores),
-                          _ptr(nhyp), _ptr(keep), _ptr(counts))
+    _load().oracle_decode_opt(_ptr(lp), T * V, V, _ptr(lengths), B, T, V, blank, K,
+                              float(np.float32(r)), int(top_n), float(beam_threshold), L,
+                              _ptr(tokens), _ptr(lens), _ptr(scores), _ptr(nhyp), _ptr(keep),
+                              _ptr(counts))
     return DecodeResult(tokens, lens, scores, nhyp,
                         None if keep is None else keep.astype(bool), counts)
 
@@ -120,9 +136,11 @@ def decode(lp: np.ndarray, lengths, blank: int, K: int, r: float, max_len: int |
 class Stream:
     """One utterance decoded incrementally; state persists between ``feed`` calls."""
 
-    def __init__(self, V: int, blank: int, K: int, r: float):
+    def __init__(self, V: int, blank: int, K: int, r: float, top_n: int = 0,
+                 beam_threshold: float = 0.0):
         self.V, self.K = V, K
         self._h = _load().oracle_stream_create(V, blank, K, float(np.float32(r)))
+        _load().oracle_stream_options(self._h, int(top_n), float(beam_threshold))
 
     def feed(self, lp: np.ndarray):
         lp = np.ascontiguousarray(lp, dtype=np.float32).reshape(-1, self.V)

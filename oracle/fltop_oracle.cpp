@@ -20,9 +20,14 @@
 // Algorithm 1 leaves out the CTC collapsing rule of the "standard
 // BeamSearchCTC decoders" it modifies (Section 3); the standard rule is used:
 // every prefix carries the log-mass of its alignments ending in blank (pb) and
-// ending in its last token (pnb).  The top-N stage (N), beam_threshold and
-// the language model of Algorithm 1 are not part of this path (N = V, no
-// threshold, no LM).
+// ending in its last token (pnb).  The language model of Algorithm 1 is not part
+// of this path.  The two remaining knobs of Algorithm 1 are optional:
+//   * N (PartialSortDesc(logits[t], N)): only the N most probable tokens of a
+//     frame are considered at all, before the relative threshold is applied;
+//     at a tie for the N-th place the lower token id wins.  top_n = 0 means N = V.
+//   * beam_threshold (second argument of SelectTopK): after the best beam_size
+//     candidates are chosen, those scoring below best - beam_threshold are
+//     dropped.  beam_threshold <= 0 means no such cut.
 //
 // A prefix is identified by its full token sequence.  Sequences are stored in
 // a trie whose child table is never pruned, so one node id corresponds to
@@ -64,6 +69,8 @@ struct TrieNode {
 
 struct Decoder {
   int V, blank, K;
+  int top_n = 0;                 // 0: no cap
+  double beam_threshold = 0.0;   // <= 0: no cut
   float log_r;
   std::vector<TrieNode> nodes;                  // node 0 = empty prefix
   std::map<std::pair<int, int>, int> child;     // (parent node, token) -> node
@@ -112,6 +119,16 @@ struct Decoder {
     for (int c = 0; c < V; ++c) {
       keep[c] = lp[c] >= thr ? 1 : 0;
       n += keep[c];
+    }
+    if (top_n > 0 && n > top_n) {
+      // stage 1 of Algorithm 1: only the top_n most probable tokens are looked at
+      std::vector<int> order;
+      for (int c = 0; c < V; ++c)
+        if (keep[c]) order.push_back(c);
+      std::stable_sort(order.begin(), order.end(),
+                       [lp](int a, int b) { return lp[a] > lp[b]; });  // ties keep id order
+      for (size_t i = top_n; i < order.size(); ++i) keep[order[i]] = 0;
+      n = top_n;
     }
     return n;
   }
@@ -163,6 +180,12 @@ struct Decoder {
       return sequence(a.node) < sequence(b.node);
     });
     if ((int)cands.size() > K) cands.resize(K);
+    if (beam_threshold > 0.0 && !cands.empty()) {
+      const double floor = cands[0].tot - beam_threshold;
+      size_t n = cands.size();
+      while (n > 1 && cands[n - 1].tot < floor) --n;
+      cands.resize(n);
+    }
     beam.clear();
     for (const auto& c : cands) beam.emplace_back(c.node, c.m);
     ++frames_seen;
@@ -184,6 +207,18 @@ void oracle_prune(const float* lp, int64_t n_frames, int V, float r, uint8_t* ke
 }
 
 void* oracle_stream_create(int V, int blank, int K, float r) { return new Decoder(V, blank, K, r); }
+// The optional knobs of Algorithm 1 (see the header of this file); call before feeding.
+void oracle_stream_options(void* h, int top_n, double beam_threshold) {
+  ((Decoder*)h)->top_n = top_n;
+  ((Decoder*)h)->beam_threshold = beam_threshold;
+}
+// Survivor mask with the top-N cap.
+void oracle_prune_topn(const float* lp, int64_t n_frames, int V, float r, int top_n, uint8_t* keep,
+                       int32_t* counts) {
+  Decoder d(V, 0, 1, r);
+  d.top_n = top_n;
+  for (int64_t t = 0; t < n_frames; ++t) counts[t] = d.prune(lp + t * V, keep + t * V);
+}
 void oracle_stream_destroy(void* h) { delete (Decoder*)h; }
 void oracle_stream_reset(void* h) { ((Decoder*)h)->reset(); }
 
@@ -224,11 +259,14 @@ int oracle_stream_results(void* h, int32_t* tokens, int32_t* lens, double* score
 // stride_t); frames t >= lengths[b] are never read.  Outputs: tokens
 // [B,K,max_len], lens [B,K], scores [B,K] (float64), nhyp [B]; optional
 // keep [B,T,V] and counts [B,T] (entries of unread frames are left untouched).
-void oracle_decode(const float* lp, int64_t stride_b, int64_t stride_t, const int32_t* lengths,
-                   int B, int T, int V, int blank, int K, float r, int max_len, int32_t* tokens,
-                   int32_t* lens, double* scores, int32_t* nhyp, uint8_t* keep, int32_t* counts) {
+void oracle_decode_opt(const float* lp, int64_t stride_b, int64_t stride_t, const int32_t* lengths,
+                       int B, int T, int V, int blank, int K, float r, int top_n,
+                       double beam_threshold, int max_len, int32_t* tokens, int32_t* lens,
+                       double* scores, int32_t* nhyp, uint8_t* keep, int32_t* counts) {
   for (int b = 0; b < B; ++b) {
     Decoder d(V, blank, K, r);
+    d.top_n = top_n;
+    d.beam_threshold = beam_threshold;
     int len = lengths[b];
     if (len < 0 || len > T) {
       nhyp[b] = 0;
@@ -245,6 +283,13 @@ void oracle_decode(const float* lp, int64_t stride_b, int64_t stride_t, const in
     nhyp[b] = oracle_stream_results(&d, tokens + (int64_t)b * K * max_len, lens + (int64_t)b * K,
                                     scores + (int64_t)b * K, nullptr, nullptr, max_len);
   }
+}
+
+void oracle_decode(const float* lp, int64_t stride_b, int64_t stride_t, const int32_t* lengths,
+                   int B, int T, int V, int blank, int K, float r, int max_len, int32_t* tokens,
+                   int32_t* lens, double* scores, int32_t* nhyp, uint8_t* keep, int32_t* counts) {
+  oracle_decode_opt(lp, stride_b, stride_t, lengths, B, T, V, blank, K, r, 0, 0.0, max_len, tokens,
+                    lens, scores, nhyp, keep, counts);
 }
 
 }  // extern "C"

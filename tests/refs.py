@@ -58,8 +58,8 @@ def _lse(a, b):
 class PyPrefixSearch:
     """Dictionary-keyed CTC prefix beam search, optional per-frame survivor sets."""
 
-    def __init__(self, blank: int, K: int):
-        self.blank, self.K = blank, K
+    def __init__(self, blank: int, K: int, beam_threshold: float = 0.0):
+        self.blank, self.K, self.beam_threshold = blank, K, beam_threshold
         self.beam = {(): (0.0, -math.inf)}
         self.revivals = 0          # prefixes that re-entered the beam after leaving it
         self._ever = {()}
@@ -85,7 +85,11 @@ class PyPrefixSearch:
                     add(seq + (c,), 1, tot + v)
         items = [(k, v) for k, v in nxt.items() if _lse(*v) > -math.inf]
         items.sort(key=lambda kv: (-_lse(*kv[1]), len(kv[0]), kv[0]))
-        self.beam = dict(items[: self.K])
+        items = items[: self.K]
+        if self.beam_threshold > 0 and items:
+            floor = _lse(*items[0][1]) - self.beam_threshold
+            items = [kv for kv in items if _lse(*kv[1]) >= floor]
+        self.beam = dict(items)
         now = set(self.beam)
         self.revivals += len([s for s in now if s in self._ever and s not in self._prev])
         self._ever |= now
@@ -97,15 +101,25 @@ class PyPrefixSearch:
         return out
 
 
-def py_decode(lp: np.ndarray, blank: int, K: int, log_r: np.float32 | None):
-    """Decode one utterance [T,V]; ``log_r`` None means no survivor test at all."""
+def top_n_tokens(row: np.ndarray, n: int):
+    """The n most probable tokens of a frame; at a tie the lower id comes first."""
+    return [int(c) for c in np.argsort(-row.astype(np.float64), kind="stable")[:n]]
+
+
+def py_decode(lp: np.ndarray, blank: int, K: int, log_r: np.float32 | None, top_n: int = 0,
+              beam_threshold: float = 0.0):
+    """Decode one utterance [T,V]; ``log_r`` None means no survivor test at all.
+
+    ``top_n`` > 0: only the top_n most probable tokens of a frame are candidates for the
+    survivor test.  ``beam_threshold`` > 0: kept prefixes score at least best - beam_threshold."""
     T, V = lp.shape
-    s = PyPrefixSearch(blank, K)
+    s = PyPrefixSearch(blank, K, beam_threshold)
     for t in range(T):
+        cand = top_n_tokens(lp[t], top_n) if top_n > 0 else range(V)
         if log_r is None:
-            surv = range(V)
+            surv = sorted(cand)
         else:
             thr = np.float32(lp[t].max()) + np.float32(log_r)
-            surv = [c for c in range(V) if lp[t, c] >= thr]
+            surv = sorted(c for c in cand if lp[t, c] >= thr)
         s.step(lp[t], surv)
     return s

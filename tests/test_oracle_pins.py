@@ -232,3 +232,87 @@ def test_empty_and_invalid_lengths():
     assert res.nhyp.tolist()[0] == 1 and res.hyps(0) == [((), 0.0)]
     assert res.nhyp[2] == 0
     assert (res.lens[0] == 0).all() and res.scores[0, 1] == -np.inf
+
+
+# ---------------------------------------------------------------- N and beam_threshold of Algorithm 1
+@pytest.mark.parametrize("V,n", [(8, 1), (8, 3), (32, 4), (32, 32), (100, 7)])
+def test_top_n_keeps_the_n_most_probable_tokens(V, n):
+    # stage 1 of Algorithm 1 against numpy's stable sort: with R = 0 the survivors are exactly
+    # the n largest entries of the row (ties: lower id), with R > 0 their intersection with
+    # the uncapped survivor set
+    lp = _rand_logp(40 + V, 30, V)
+    lp[3, :] = lp[3, 0]                      # a row of exact ties: ids 0 .. n-1 must win
+    lp[4, 2] = lp[4, 5] = lp[4].max() + 1.0  # a tie for first place
+    keep, cnt = oracle.prune(lp, 0.0, top_n=n)
+    for t in range(lp.shape[0]):
+        want = np.zeros(V, dtype=bool)
+        want[np.argsort(-lp[t].astype(np.float64), kind="stable")[:n]] = True
+        assert (keep[t] == want).all() and cnt[t] == min(n, V)
+    keep_r, _ = oracle.prune(lp, 0.05)
+    keep_rn, cnt_rn = oracle.prune(lp, 0.05, top_n=n)
+    keep_n, _ = oracle.prune(lp, 0.0, top_n=n)
+    assert (keep_rn == (keep_r & keep_n)).all()
+    assert (cnt_rn <= n).all() and keep_rn[np.arange(30), lp.argmax(1)].all()
+    # n >= V and n = 0 change nothing
+    assert (oracle.prune(lp, 0.05, top_n=V)[0] == keep_r).all()
+    assert (oracle.prune(lp, 0.05, top_n=0)[0] == keep_r).all()
+
+
+@pytest.mark.parametrize("seed,T,V,n,r", [(0, 5, 4, 2, 0.0), (1, 6, 3, 1, 0.0), (2, 5, 4, 3, 0.2)])
+def test_top_n_inside_the_search_is_brute_force_over_the_kept_tokens(seed, T, V, n, r):
+    lp = _rand_logp(seed + 70, T, V)
+    keep = np.zeros((T, V), dtype=bool)
+    for t in range(T):
+        keep[t, np.argsort(-lp[t].astype(np.float64), kind="stable")[:n]] = True
+        if r > 0:
+            keep[t] &= lp[t] >= np.float32(lp[t].max()) + oracle.log_r(r)
+    exact = {k: v for k, v in brute_force(lp, 0, keep).items() if v > -math.inf}
+    res = oracle.decode(lp[None], [T], 0, 4096, r, top_n=n, want_masks=True)
+    assert (res.keep[0] == keep).all()
+    got = dict(res.hyps(0))
+    assert set(got) == set(exact)
+    for k, v in exact.items():
+        assert got[k] == pytest.approx(v, abs=1e-9)
+
+
+def test_top_n_one_is_greedy_whatever_the_beam():
+    lp = _rand_logp(5, 60, 12)
+    for K in (1, 5):
+        res = oracle.decode(lp[None], [60], 0, K, 0.0, top_n=1)
+        assert res.hyps(0)[0][0] == greedy(lp, 0)
+        assert res.nhyp[0] == 1          # one token per frame: one prefix
+
+
+@pytest.mark.parametrize("K,theta,r,n", [(6, 2.0, 0.0, 0), (10, 0.5, 0.05, 0), (8, 4.0, 0.01, 3),
+                                         (4, 1e-9, 0.0, 0)])
+def test_beam_threshold_and_top_n_match_the_second_implementation(K, theta, r, n):
+    for seed in range(4):
+        lp = _rand_logp(200 + seed, 40, 6, sharp=1.0)
+        ref = py_decode(lp, 0, K, None if r == 0 else oracle.log_r(r), top_n=n,
+                        beam_threshold=theta).results()
+        got = oracle.decode(lp[None], [40], 0, K, r, top_n=n, beam_threshold=theta).hyps(0)
+        assert [s for s, _ in got] == [s for s, _ in ref]
+        np.testing.assert_allclose([v for _, v in got], [v for _, v in ref], atol=1e-9)
+
+
+def test_beam_threshold_invariants():
+    lp = _rand_logp(9, 80, 8, sharp=3.0)
+    base = oracle.decode(lp[None], [80], 0, 12, 0.01).hyps(0)
+    # off, and a threshold nothing can reach, change nothing
+    assert oracle.decode(lp[None], [80], 0, 12, 0.01, beam_threshold=0.0).hyps(0) == base
+    assert oracle.decode(lp[None], [80], 0, 12, 0.01, beam_threshold=1e9).hyps(0) == base
+    for theta in (8.0, 3.0, 1.0, 0.2, 0.01):
+        h = oracle.decode(lp[None], [80], 0, 12, 0.01, beam_threshold=theta).hyps(0)
+        assert all(s >= h[0][1] - theta for _, s in h) and 1 <= len(h) <= 12
+    # a vanishing threshold leaves the single best prefix of every frame: the K = 1 search
+    one = oracle.decode(lp[None], [80], 0, 12, 0.01, beam_threshold=1e-12).hyps(0)
+    assert len(one) == 1 and one == oracle.decode(lp[None], [80], 0, 1, 0.01).hyps(0)
+
+
+def test_streaming_with_options_equals_one_shot():
+    lp = _rand_logp(31, 50, 10, sharp=1.0)
+    full = oracle.decode(lp[None], [50], 0, 6, 0.02, top_n=4, beam_threshold=3.0).hyps(0)
+    st = oracle.Stream(10, 0, 6, 0.02, top_n=4, beam_threshold=3.0)
+    for a, b in [(0, 7), (7, 8), (8, 33), (33, 50)]:
+        st.feed(lp[a:b])
+    assert st.results() == full
