@@ -368,11 +368,11 @@ def run_report(args):
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     rows = []
 
-    def measure(wl, K, r, label, top1_ref=None):
+    def measure(wl, K, r, label, top1_ref=None, top_n=0, theta=0.0):
         B, T, V = wl.emissions.shape
         x = torch.from_numpy(wl.emissions).cuda()
         ln = torch.from_numpy(wl.lengths).cuda()
-        dec = binding.Decoder(V, wl.blank_id, K, r, B, T)
+        dec = binding.Decoder(V, wl.blank_id, K, r, B, T, top_n=top_n, beam_threshold=theta)
         dec.set_profiling(True)
         ms, pk, dk = _time_decode(dec, x, ln, flush)
         st = dec.last_call_stats()
@@ -411,6 +411,13 @@ def run_report(args):
               file=sys.stderr, flush=True)
         for r in workloads.SWEEP_THRESHOLDS:
             measure(wav, K, r, "2 sweep", ref)
+    # the paper's own operating point (Sections 4.2-4.4): N = 4, R = 0.007, beam_threshold = 25,
+    # against its baseline (all tokens, same beam_threshold) and Top-4 without R
+    for K in (50, 1000):
+        ref = None if args.skip_oracle or K > 50 else _oracle_top1(wav, K, 0.0, cores)
+        measure(wav, K, 0.0, "P baseline (all tokens, bt 25)", ref, theta=25.0)
+        measure(wav, K, 0.0, "P Top-4 (bt 25)", ref, top_n=4, theta=25.0)
+        measure(wav, K, 0.007, "P FLToP N=4 R=0.007 (bt 25)", ref, top_n=4, theta=25.0)
     sub = workloads.workload_subword()
     for r in sub.thresholds:
         measure(sub, sub.beam_width, r, "3 subword")

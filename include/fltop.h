@@ -11,8 +11,8 @@
  * whole beam).  The CTC collapsing rule is the standard one of the "standard
  * BeamSearchCTC decoders" the paper modifies (Section 3): each prefix carries
  * the log-mass of alignments ending in blank and ending in its last token.
- * The top-N stage, beam_threshold and the language model of Algorithm 1 are
- * not implemented (their config fields are reserved).
+ * The top-N stage (N) and beam_threshold of Algorithm 1 are optional config
+ * fields; its language model is not implemented.
  *
  * Conventions
  *   - every `d_*` pointer is DEVICE memory owned by the caller; the library
@@ -71,8 +71,13 @@ typedef struct {
   int32_t max_chunk_frames; /* 0: the handle serves fltop_decode.  > 0: the handle serves
                              fltop_stream_step with chunks of at most this many frames */
   int32_t max_out_len;    /* L of the token output, 1 <= L */
-  int32_t top_n;          /* reserved (N of Algorithm 1); must be 0 */
-  float beam_threshold;   /* reserved (beam_threshold of Algorithm 1); must be <= 0 */
+  int32_t top_n;          /* N of Algorithm 1 (PartialSortDesc): a frame keeps at most its
+                             top_n most probable tokens, before R is applied; at a tie for
+                             the last place the lower token id stays.  0 = no cap */
+  float beam_threshold;   /* beam_threshold of Algorithm 1 (SelectTopK): of the beam_width
+                             best prefixes of a frame, those scoring below best -
+                             beam_threshold are dropped, so a beam can hold fewer than
+                             beam_width prefixes.  <= 0 = no such cut */
   int32_t device;         /* CUDA device ordinal */
   void* workspace;        /* optional DEVICE memory, 256-byte aligned, for all of the
                              handle's scratch; NULL = the library allocates it */

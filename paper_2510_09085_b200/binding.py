@@ -161,9 +161,10 @@ class Decoder:
     """Owns one handle plus the output tensors; thin convenience over the C calls."""
 
     def __init__(self, vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
-                 max_chunk_frames=0, max_out_len=None, device=0):
+                 max_chunk_frames=0, max_out_len=None, device=0, top_n=0, beam_threshold=0.0):
         self.cfg = make_config(vocab_size, blank_id, beam_width, threshold_r, max_batch,
-                               max_frames, max_chunk_frames, max_out_len, device)
+                               max_frames, max_chunk_frames, max_out_len, device, top_n=top_n,
+                               beam_threshold=beam_threshold)
         code, self.h = fltop_create(self.cfg)
         if code != FLTOP_OK:
             self.h = None

@@ -49,8 +49,8 @@ bool config_ok(const fltop_config* c) {
   if (!(c->threshold_r >= 0.f && c->threshold_r <= 1.f)) return false;  // rejects NaN too
   if (c->max_batch < 1 || c->max_frames < 1 || c->max_out_len < 1) return false;
   if (c->max_chunk_frames < 0 || c->max_chunk_frames > c->max_frames) return false;
-  if (c->top_n != 0) return false;
-  if (c->beam_threshold > 0.f || c->beam_threshold != c->beam_threshold) return false;
+  if (c->top_n < 0) return false;
+  if (c->beam_threshold != c->beam_threshold) return false;  // NaN
   if (c->device < 0) return false;
   if ((int64_t)(c->beam_width + 1) * c->max_frames + 2 > (int64_t)std::numeric_limits<int32_t>::max())
     return false;
@@ -125,6 +125,7 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.K = h->cfg.beam_width; dp.blank = h->cfg.blank_id; dp.L = h->cfg.max_out_len;
   dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
   dp.block_threads = h->block_threads; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
+  dp.top_n = h->cfg.top_n; dp.beam_threshold = h->cfg.beam_threshold;
   dp.counts = h->counts; dp.entries = h->entries; dp.nodes = h->nodes;
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
@@ -137,6 +138,11 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
     e = launch_prune(pp, s);
     if (e != cudaSuccess) return cuda_fail(h, e);
     ++h->launches;
+    if (h->cfg.top_n > 0 && h->cfg.top_n < h->cfg.vocab_size) {
+      e = launch_topn_cap(pp, h->cfg.top_n, s);
+      if (e != cudaSuccess) return cuda_fail(h, e);
+      ++h->launches;
+    }
   }
   if (h->profiling) cudaEventRecord(h->ev[1], s);
   e = launch_decode(dp, s);
@@ -271,6 +277,11 @@ int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t 
   e = launch_prune(pp, static_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) return cuda_fail(h, e);
   ++h->launches;
+  if (h->cfg.top_n > 0 && h->cfg.top_n < h->cfg.vocab_size) {
+    e = launch_topn_cap(pp, h->cfg.top_n, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    ++h->launches;
+  }
   return FLTOP_OK;
 }
 

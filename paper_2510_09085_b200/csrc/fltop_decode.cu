@@ -181,10 +181,10 @@ struct __align__(16) FrameInfo {
 
 enum {
   // one copy per frame parity
-  SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_PER_FRAME,
+  SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_MAXKEY, SC_PER_FRAME,
   // single copies
   SC_THR = 2 * SC_PER_FRAME, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_TOTAL, SC_FIRST, SC_STATUS,
-  SC_CREATED,
+  SC_CREATED, SC_DEAD, SC_NLIVE,
   // exact fallback select
   SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_NBEAM_NEXT, SC_COUNT
 };
@@ -382,7 +382,8 @@ __device__ __forceinline__ void divmod_small(int e, int d, float inv_d, int& q, 
 // KMAX / VMAX > 0: the shared-memory arrays are laid out for that beam width and vocabulary
 // whatever K and V are (K <= KMAX, V <= VMAX), so every array offset is a compile-time
 // constant; 0: laid out for the K and V of the call.
-template <int MAXT, int KMAX, int VMAX>
+// BT: beam_threshold is on (the exact best score of every frame is tracked).
+template <int MAXT, int KMAX, int VMAX, bool BT>
 __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
@@ -430,6 +431,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   const bool is_ext = !is_chore && !is_stay;
   const int xl = tid - NS;                   // index among the ext lanes
   const bool warp_scans = NT <= kSmallBlock;
+  constexpr bool use_bt = BT;
 
   int len = p.lengths[b];
   unsigned flags = 3u;
@@ -659,8 +661,12 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     float kc[kCache];  // this ext lane's first extension scores (-inf: none)
 #pragma unroll
     for (int k = 0; k < kCache; ++k) kc[k] = neg_inf();
+    float my_max = neg_inf();  // best score among this thread's candidates (beam_threshold only)
     if (is_stay) {
-      for (int i = tid; i < nb; i += NS) stay_eval(i);
+      for (int i = tid; i < nb; i += NS) {
+        const float sc = stay_eval(i);
+        if (use_bt) my_max = fmaxf(my_max, sc);
+      }
     } else if (is_ext) {
       divmod_small(xl, Sdiv, fi.inv_s, q0, j0);
       int q = q0, j = j0;
@@ -670,12 +676,14 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           const float sc = ext_score(hc[q], j);
           step(q, j);
           kc[k] = sc;
+          if (use_bt) my_max = fmaxf(my_max, sc);
           if (sc != neg_inf()) count(sc);
         }
       }
       for (int e = xl + kCache * NX; e < next; e += NX) {
         const float sc = ext_score(hc[q], j);
         step(q, j);
+        if (use_bt) my_max = fmaxf(my_max, sc);
         if (sc != neg_inf()) count(sc);
       }
     } else {
@@ -704,7 +712,15 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         sc_n[SC_LISTN] = 0;
         sc_n[SC_SLOT] = 0;
         sc_n[SC_SLOT_E] = 0;
+        sc_n[SC_MAXKEY] = 0;
       }
+    }
+    if (use_bt && !is_chore) {
+      // SelectTopK's beam_threshold is relative to the exact best score of the frame
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) my_max = fmaxf(my_max, __shfl_xor_sync(kFull, my_max, o));
+      if (lane == 0 && my_max != neg_inf())
+        atomicMax(reinterpret_cast<unsigned*>(&sc_c[SC_MAXKEY]), score_key(my_max));
     }
     __syncthreads();  // B1
 
@@ -756,6 +772,21 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     const bool take_all = cut.cut_count == cut.left;  // also true when there is no cut at all
     const bool use_list = !take_all && cut.cut_count <= kListCap;
     int nbn = min(cut.total, K);
+    // beam_threshold: a selected candidate scoring below (best of the frame) - threshold is
+    // dropped.  Its beam slot is written as a dead entry (probability 0, no identity).
+    float f_floor = neg_inf();
+    if (use_bt) {
+      const unsigned mk = (unsigned)sc_c[SC_MAXKEY];
+      if (mk) f_floor = key_score(mk) - p.beam_threshold;
+    }
+    auto place_dead = [&](int slot) {
+      Hot e;
+      e.last = -1; e.pb = e.pnb = e.tot = neg_inf();
+      hn[slot] = e;
+      id_n[slot] = Ident{0ull, 0ull};
+      wh_n[slot] = Where{0, 0};
+      atomicAdd(&scal[SC_DEAD], 1);
+    };
     TrieNode* const nst = nstage + par * NSL;
     // the frame's nodes get ids n_nodes .. n_nodes + nbn - 1 (the slots of stays stay unused)
     const bool arena_ok = (int64_t)n_nodes + ((K + 1) & ~1) <= p.nodes_per_utt;
@@ -763,6 +794,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     // ---- P3: selected candidates take their slots in the next beam ---------------------
     auto place_stay = [&](int q, unsigned key, int slot) {
       if ((unsigned)slot >= (unsigned)K) return;  // only reachable with NaN scores
+      if (use_bt && key_score(key) < f_floor) return place_dead(slot);
       Hot e;
       e.last = hc[q].last;
       e.pb = st_pb[q] - best;
@@ -776,6 +808,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     };
     auto place_ext = [&](int q, int tok, unsigned key, int slot) {
       if ((unsigned)slot >= (unsigned)K) return;
+      if (use_bt && key_score(key) < f_floor) return place_dead(slot);
       const float sc = key_score(key) - best;
       Hot e;
       e.last = tok; e.pb = neg_inf(); e.pnb = sc; e.tot = sc;
@@ -995,7 +1028,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     __syncthreads();
     if (tid == 0) {
       int32_t* o = p.stats + 4 * (int64_t)b;
-      o[0] = len; o[1] = scal[SC_CREATED]; o[2] = live_sum; o[3] = n_nodes;
+      o[0] = len; o[1] = scal[SC_CREATED]; o[2] = live_sum - scal[SC_DEAD]; o[3] = n_nodes;
     }
   }
 
@@ -1030,6 +1063,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     bool truncated = false;
     for (int i = tid; i < nb; i += NT) {
       const float ti = hc[i].tot;
+      if (ti == neg_inf()) continue;  // a slot emptied by beam_threshold
+      atomicAdd(&scal[SC_NLIVE], 1);
       int rank = 0;
       for (int j = 0; j < nb; ++j) {
         const float tj = hc[j].tot;
@@ -1049,14 +1084,15 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         node = rec.x;
       }
     }
-    for (int k = nb + tid; k < K; k += NT) {
+    if (truncated) atomicOr(&scal[SC_STATUS], 4);  // FLTOP_ST_TRUNCATED
+    __syncthreads();
+    const int n_live = scal[SC_NLIVE];
+    for (int k = n_live + tid; k < K; k += NT) {
       p.out_lens[(int64_t)b * K + k] = 0;
       p.out_scores[(int64_t)b * K + k] = neg_inf();
     }
-    if (truncated) atomicOr(&scal[SC_STATUS], 4);  // FLTOP_ST_TRUNCATED
-    __syncthreads();
     status |= scal[SC_STATUS];
-    if (tid == 0) p.out_nhyp[b] = nb;
+    if (tid == 0) p.out_nhyp[b] = n_live;
   }
   if (tid == 0 && p.out_status) p.out_status[b] = status;
 }
@@ -1080,7 +1116,7 @@ size_t decode_smem_bytes(int K, int V) {
   }
 }
 
-int decode_block_threads(int K, int V, bool pruning) {
+int decode_block_threads(int K, int V, bool pruning, int top_n) {
   // one lane per beam entry for the stay candidates, about three extension candidates per
   // ext lane, one chore warp.  With pruning on, a quarter of a large vocabulary (at least
   // eight tokens) is assumed to survive a frame.
@@ -1090,6 +1126,7 @@ int decode_block_threads(int K, int V, bool pruning) {
     if (cols < 8) cols = 8;
     if (cols > V) cols = V;
   }
+  if (top_n > 0 && top_n < cols) cols = top_n;
   const long long stay = ((long long)K + 31) / 32 * 32;
   long long ext = ((long long)K * cols / 3 + 31) / 32 * 32;
   if (ext < 32) ext = 32;
@@ -1101,16 +1138,23 @@ int decode_block_threads(int K, int V, bool pruning) {
 namespace {
 template <int KMAX, int VMAX>
 cudaError_t prepare_variant(int bytes) {
-  cudaError_t e = cudaFuncSetAttribute(decode_kernel<kSmallBlock, KMAX, VMAX>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  cudaError_t e = cudaFuncSetAttribute(decode_kernel<kSmallBlock, KMAX, VMAX, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kSmallBlock, KMAX, VMAX, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX, true>, attr, bytes);
+  return e;
 }
 template <int KMAX, int VMAX>
 void launch_variant(const DecodeParams& p, int nt, size_t bytes, cudaStream_t s) {
-  if (nt <= kSmallBlock) decode_kernel<kSmallBlock, KMAX, VMAX><<<p.B, nt, bytes, s>>>(p);
-  else decode_kernel<kMaxThreads, KMAX, VMAX><<<p.B, nt, bytes, s>>>(p);
+  const bool bt = p.beam_threshold > 0.f;
+  if (nt <= kSmallBlock) {
+    if (bt) decode_kernel<kSmallBlock, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
+    else decode_kernel<kSmallBlock, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
+  } else {
+    if (bt) decode_kernel<kMaxThreads, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
+    else decode_kernel<kMaxThreads, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
+  }
 }
 }  // namespace
 
@@ -1125,7 +1169,7 @@ cudaError_t decode_prepare(int K, int V) {
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   if (p.B == 0) return cudaSuccess;
-  int nt = p.block_threads > 0 ? p.block_threads : decode_block_threads(p.K, p.V, p.pruning != 0);
+  int nt = p.block_threads > 0 ? p.block_threads : decode_block_threads(p.K, p.V, p.pruning != 0, p.top_n);
   nt = (nt + 31) / 32 * 32;
   if (nt < 96) nt = 96;  // a stay warp, an ext warp and the chore warp
   if (nt > kMaxThreads) nt = kMaxThreads;

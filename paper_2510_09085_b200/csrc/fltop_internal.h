@@ -52,6 +52,8 @@ struct DecodeParams {
   int32_t emit_default;     // streaming with flags == null: emit results?
   int32_t block_threads;    // 0 = choose from K, V and whether pruning is on
   int32_t pruning;          // 1 when R is large enough that few tokens survive a frame
+  int32_t top_n;            // survivors per frame are capped at this (0: no cap)
+  float beam_threshold;     // kept prefixes score at least best - beam_threshold (<= 0: off)
   const int32_t* counts;    // [B*T] survivors per frame
   const Survivor* entries;  // [B*T*V]
   TrieNode* nodes;          // [B * nodes_per_utt]
@@ -66,8 +68,10 @@ struct DecodeParams {
 };
 
 size_t decode_smem_bytes(int K, int V);
-int decode_block_threads(int K, int V, bool pruning);
+int decode_block_threads(int K, int V, bool pruning, int top_n);
 cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
+// keeps at most top_n survivors per frame (no-op for top_n <= 0 or >= V)
+cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s);
 cudaError_t decode_prepare(int K, int V);  // one-time kernel attribute set-up
 

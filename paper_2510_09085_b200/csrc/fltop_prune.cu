@@ -126,6 +126,88 @@ __global__ void __launch_bounds__(kPruneThreads) prune_scalar_kernel(PruneParams
   }
 }
 
+// Stage 1 of Algorithm 1 (PartialSortDesc(logits[t], N)): a frame keeps at most its top_n most
+// probable survivors; at a tie for the last place the lower token id wins.  One warp per
+// frame that has more than top_n survivors: an 8-bit radix select over order-preserving
+// integer keys finds the top_n-th largest log-probability, then the list is compacted in
+// place (it stays in ascending token order).
+__global__ void __launch_bounds__(kPruneThreads) topn_cap_kernel(PruneParams p, int top_n) {
+  __shared__ unsigned hist_all[kPruneThreads / 32][256];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned* const h = hist_all[warp];
+  const unsigned lt_mask = (1u << lane) - 1u;
+  const int64_t n_rows = (int64_t)p.B * p.T;
+  const int64_t warp_global = (int64_t)blockIdx.x * (kPruneThreads / 32) + warp;
+  const int64_t warp_stride = (int64_t)gridDim.x * (kPruneThreads / 32);
+  auto order_key = [](float v) -> unsigned {
+    const unsigned u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  };
+  for (int64_t row = warp_global; row < n_rows; row += warp_stride) {
+    const int count = p.counts[row];
+    if (count <= top_n) continue;  // warp-uniform
+    Survivor* const list = p.entries + row * p.V;
+    unsigned prefix = 0u;
+    int need = top_n;  // how many of the keys that share `prefix` are still to be taken
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      for (int i = lane; i < 256; i += 32) h[i] = 0u;
+      __syncwarp();
+      for (int i = lane; i < count; i += 32) {
+        const unsigned key = order_key(list[i].logp);
+        if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&h[(key >> shift) & 255u], 1u);
+      }
+      __syncwarp();
+      // lane l owns digits 255 - 8l .. 248 - 8l, walked from the largest
+      unsigned c = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) c += h[255 - (lane * 8 + i)];
+      unsigned inc = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+      }
+      const unsigned hit = __ballot_sync(0xffffffffu, (int)inc >= need);
+      const int owner = __ffs(hit) - 1;  // exists: the group holds at least `need` keys
+      int digit = 0, left = 0;
+      if (lane == owner) {
+        unsigned acc = inc - c;
+        digit = 255 - lane * 8;
+        for (int i = 0; i < 8; ++i, --digit) {
+          const unsigned n = h[digit];
+          if ((int)(acc + n) >= need) break;
+          acc += n;
+        }
+        left = need - (int)acc;
+      }
+      digit = __shfl_sync(0xffffffffu, digit, owner);
+      need = __shfl_sync(0xffffffffu, left, owner);
+      prefix = (prefix << 8) | (unsigned)digit;
+      __syncwarp();
+    }
+    // keys above `prefix` all stay; of the keys equal to it, the first `need` in token order
+    int out_pos = 0, eq_seen = 0;
+    for (int base = 0; base < count; base += 32) {
+      const int i = base + lane;
+      Survivor s = Survivor{0, 0.f};
+      unsigned key = 0u;
+      if (i < count) {
+        s = list[i];
+        key = order_key(s.logp);
+      }
+      const bool eq = i < count && key == prefix;
+      const unsigned eqm = __ballot_sync(0xffffffffu, eq);
+      const bool keep = i < count && (key > prefix || (eq && eq_seen + __popc(eqm & lt_mask) < need));
+      const unsigned km = __ballot_sync(0xffffffffu, keep);  // every lane has loaded its entry
+      if (keep) list[out_pos + __popc(km & lt_mask)] = s;
+      out_pos += __popc(km);
+      eq_seen += __popc(eqm);
+    }
+    if (lane == 0) p.counts[row] = out_pos;
+  }
+}
+
 template <int LPR, int CH>
 cudaError_t launch_vec(const PruneParams& p, cudaStream_t s, int sms) {
   const int64_t n_rows = (int64_t)p.B * p.T;
@@ -164,6 +246,18 @@ cudaError_t launch_prune(const PruneParams& p, cudaStream_t s) {
   int64_t blocks = (n_rows + (kPruneThreads / 32) - 1) / (kPruneThreads / 32);
   if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
   prune_scalar_kernel<<<(unsigned)blocks, kPruneThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s) {
+  const int64_t n_rows = (int64_t)p.B * p.T;
+  if (n_rows == 0 || top_n <= 0 || top_n >= p.V) return cudaSuccess;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int64_t blocks = (n_rows + (kPruneThreads / 32) - 1) / (kPruneThreads / 32);
+  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+  topn_cap_kernel<<<(unsigned)blocks, kPruneThreads, 0, s>>>(p, top_n);
   return cudaGetLastError();
 }
 
