@@ -147,6 +147,33 @@ __global__ void __launch_bounds__(kPruneThreads) topn_cap_kernel(PruneParams p, 
     const int count = p.counts[row];
     if (count <= top_n) continue;  // warp-uniform
     Survivor* const list = p.entries + row * p.V;
+    if (count <= 32 && top_n <= 8) {
+      // short list, small N: one entry per lane, the best one leaves top_n times (a tie goes
+      // to the earlier entry, i.e. the lower token id)
+      Survivor s = Survivor{0, 0.f};
+      unsigned long long mine = 0ull;  // 0 = not in the running
+      if (lane < count) {
+        s = list[lane];
+        mine = ((unsigned long long)order_key(s.logp) << 8) | (unsigned)(63 - lane);
+      }
+      bool keep = false;
+      for (int n = 0; n < top_n; ++n) {
+        unsigned long long best = mine;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+          best = other > best ? other : best;
+        }
+        if (mine == best) {
+          keep = true;
+          mine = 0ull;
+        }
+      }
+      const unsigned km = __ballot_sync(0xffffffffu, keep);
+      if (keep) list[__popc(km & lt_mask)] = s;
+      if (lane == 0) p.counts[row] = __popc(km);
+      continue;
+    }
     unsigned prefix = 0u;
     int need = top_n;  // how many of the keys that share `prefix` are still to be taken
     for (int pass = 0; pass < 4; ++pass) {
