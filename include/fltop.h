@@ -59,7 +59,9 @@ enum {
 };
 
 typedef struct {
-  int32_t vocab_size;     /* V, 2 <= V <= 8192 */
+  int32_t vocab_size;     /* V, 2 <= V <= 8192; V and K together must fit one SM's shared
+                             memory (about 48 V + 130 K bytes <= 227 KB: V = 4096 with small
+                             beams, K = 1500 at V = 32), else fltop_create refuses */
   int32_t blank_id;       /* 0 <= blank_id < V */
   int32_t beam_width;     /* K = beam_size of Algorithm 1, 1 <= K <= 2048 */
   float threshold_r;      /* R of Algorithm 1 in the probability domain, 0 <= R <= 1;

@@ -284,3 +284,11 @@ def test_large_vocabulary_prefixes_leave_and_reenter():
     assert revivals > 0
     compare_batch(em, ln, 0, 4, 0.05)
     compare_batch(em, ln, 0, 3, 0.0)
+
+
+@pytest.mark.parametrize("V,K,r", [(32, 1024, 0.0), (32, 1500, 1e-3), (4096, 4, 1e-3), (2048, 16, 0.0)])
+def test_largest_shapes_fit_and_match(V, K, r):
+    # beam widths and vocabularies near what one SM's shared memory holds (generic layout,
+    # radix fallback for the wide beams), on short utterances so that the oracle stays quick
+    em, ln = W.make_small(4000 + V + K, 2, 6, 14, V)
+    compare_batch(em, ln, 0, K, r, max_unmatched_frac=0.25)
