@@ -1170,6 +1170,14 @@ cudaError_t decode_prepare(int K, int V) {
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   if (p.B == 0) return cudaSuccess;
   int nt = p.block_threads > 0 ? p.block_threads : decode_block_threads(p.K, p.V, p.pruning != 0, p.top_n);
+  if (p.block_threads <= 0 && nt > 512 && p.pruning) {
+    // more utterances than SMs: two blocks of 512 threads per SM overlap their frame chains
+    // better than one block of 1024 (measured on the subword shape, B = 256)
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (p.B > sms) nt = 512;
+  }
   nt = (nt + 31) / 32 * 32;
   if (nt < 96) nt = 96;  // a stay warp, an ext warp and the chore warp
   if (nt > kMaxThreads) nt = kMaxThreads;
