@@ -204,7 +204,7 @@ __host__ __device__ inline int node_stage_len(int K) { return (K + 1) & ~1; }
 
 // Byte offsets of the shared-memory arrays.
 struct Lay {
-  unsigned sv, hot, ident, where, nstage, finfo, warp_sums, st_pb, st_pnb, st_key, dup, tab, lpv,
+  unsigned sv, hot, ident, where, nstage, finfo, warp_sums, st_pb, st_pnb, st_tot, dup, tab, lpv,
       jpos, hist,
       rhist, list_key, list_id, sel_key, sel_id, scal, total;
 };
@@ -226,7 +226,7 @@ __host__ __device__ inline Lay make_layout(int K, int V) {
   l.warp_sums = take(34 * 8);
   l.st_pb = take(K * 4);
   l.st_pnb = take(K * 4);
-  l.st_key = take(K * 4);
+  l.st_tot = take(K * 4);
   l.dup = take(2u * dup_words(K, V) * 4);
   l.tab = take(2u * table_size(K) * 4);
   l.lpv = take(2u * V * 4);
@@ -405,7 +405,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   unsigned long long* const warp_sums = reinterpret_cast<unsigned long long*>(smem + L.warp_sums);
   float* const st_pb = reinterpret_cast<float*>(smem + L.st_pb);
   float* const st_pnb = reinterpret_cast<float*>(smem + L.st_pnb);
-  float* const st_tot = reinterpret_cast<float*>(smem + L.st_key);  // lse(st_pb, st_pnb)
+  float* const st_tot = reinterpret_cast<float*>(smem + L.st_tot);  // lse(st_pb, st_pnb)
   unsigned* const dup_base = reinterpret_cast<unsigned*>(smem + L.dup);
   TrieNode* const nstage = reinterpret_cast<TrieNode*>(smem + L.nstage);
   int* const jpos_base = reinterpret_cast<int*>(smem + L.jpos);
