@@ -184,7 +184,7 @@ enum {
   SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_MAXKEY, SC_PER_FRAME,
   // single copies
   SC_THR = 2 * SC_PER_FRAME, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_TOTAL, SC_FIRST, SC_STATUS,
-  SC_CREATED, SC_DEAD, SC_NLIVE,
+  SC_CREATED, SC_DEAD, SC_NLIVE, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL,
   // exact fallback select
   SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_NBEAM_NEXT, SC_COUNT
 };
@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   for (int i = tid; i < 2 * TS; i += NT) tab_base[i] = kEmptySlot;
   for (int i = tid; i < 2 * VS; i += NT) lpv_base[i] = neg_inf();
   for (int i = tid; i < 2 * kFastBins; i += NT) hist_base[i] = 0u;
-  if (tid < SC_COUNT) scal[tid] = 0;
+  if (tid < SC_COUNT) scal[tid] = tid == SC_NEXT_BJ ? -1 : 0;
   int created = 0, live_sum = 0;
   int cur = 0, nb, n_nodes, frames_seen;
   double offset;
@@ -520,46 +520,41 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   auto svbuf = [&](int t) -> Survivor* { return sv_base + (t & 3) * VS; };
   auto lpvbuf = [&](int t) -> float* { return lpv_base + (t & 1) * VS; };
 
-  // Chore warp: the log-probability table and the constants of frame t1 (its survivors are
-  // in shared memory), and the table of frame t1 - 1 forgotten (t1 > 0).
-  auto stage_frame = [&](int t1, int S_prev, int S1) {
+  // The tables of frame t1 (its survivors are in shared memory): token -> log-probability and
+  // token -> position in the survivor list; the table of frame t1 - 1 is forgotten (t1 > 0).
+  // Threads first, first + stride, ... share the work; whoever meets blank notes where.
+  auto stage_tables = [&](int t1, int S_prev, int S1, int first, int stride) {
     if (t1 > 0) {
       float* lp_old = lpvbuf(t1 - 1);
       const Survivor* so = svbuf(t1 - 1);
-      for (int j = lane; j < S_prev; j += 32) lp_old[so[j].token] = neg_inf();
+      for (int j = first; j < S_prev; j += stride) lp_old[so[j].token] = neg_inf();
     }
     float* lp_new = lpvbuf(t1);
-    const Survivor* sn = svbuf(t1);
-    int bj = -1;
-    float bl = neg_inf();
-    for (int j0 = 0; j0 < S1; j0 += 32) {
-      const int j = j0 + lane;
-      bool is_blank = false;
-      float lp = neg_inf();
-      if (j < S1) {
-        const Survivor s = sn[j];
-        lp_new[s.token] = s.logp;
-        is_blank = s.token == blank;
-        lp = s.logp;
-      }
-      const unsigned m = __ballot_sync(kFull, is_blank);
-      if (m) {
-        const int src = __ffs(m) - 1;
-        bj = j0 + src;
-        bl = __shfl_sync(kFull, lp, src);
-      }
-    }
     int* jp_new = jpos_base + (t1 & 1) * VS;
-    for (int j = lane; j < S1; j += 32) jp_new[sn[j].token] = j - ((bj >= 0 && j > bj) ? 1 : 0);
-    if (lane == 0) {
-      FrameInfo f;
-      f.S = S1; f.blank_j = bj; f.Snb = S1 - (bj >= 0 ? 1 : 0); f.lp_blank = bl;
-      const int d = max(f.Snb, 1);
-      f.inv_s = 1.f / (float)d;
-      divmod_small(NX, d, f.inv_s, f.dq, f.dj);
-      f.pad = 0;
-      finfo[t1 & 1] = f;
+    const Survivor* sn = svbuf(t1);
+    for (int j = first; j < S1; j += stride) {
+      const Survivor s = sn[j];
+      lp_new[s.token] = s.logp;
+      jp_new[s.token] = j;
+      if (s.token == blank) {
+        scal[SC_NEXT_BJ] = j;
+        scal[SC_NEXT_BL] = __float_as_int(s.logp);
+      }
     }
+  };
+  // One thread, once the tables of frame t1 are complete: the constants of the frame.
+  auto publish_frame = [&](int t1, int S1) {
+    FrameInfo f;
+    f.S = S1;
+    f.blank_j = scal[SC_NEXT_BJ];
+    f.lp_blank = f.blank_j >= 0 ? __int_as_float(scal[SC_NEXT_BL]) : neg_inf();
+    f.Snb = S1 - (f.blank_j >= 0 ? 1 : 0);
+    const int d = max(f.Snb, 1);
+    f.inv_s = 1.f / (float)d;
+    divmod_small(NX, d, f.inv_s, f.dq, f.dj);
+    f.pad = 0;
+    finfo[t1 & 1] = f;
+    scal[SC_NEXT_BJ] = -1;
   };
 
   // ---- prologue: survivors of frames 0 and 1, tables of frame 0 ----------------------
@@ -575,7 +570,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     cp_async_commit();
     cp_async_wait_all();
     __syncwarp();
-    stage_frame(0, 0, c0);
+    stage_tables(0, 0, c0, lane, 32);
+    __syncwarp();
+    if (lane == 0) publish_frame(0, c0);
   }
   __syncthreads();
 
@@ -631,7 +628,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           if (dup != neg_inf()) {  // the parent's extension by last(q) names this prefix
             npnb = lse2(npnb, dup);
             atomicSub(&hist[score_bin(dup)], 1u);
-            const int ed = pq * Snb + jpos[e.last];
+            const int jp = jpos[e.last];  // position among all survivors -> among non-blank
+            const int ed = pq * Snb + jp - ((blank_j >= 0 && jp > blank_j) ? 1 : 0);
             atomicOr(&dupbits[ed >> 5], 1u << (ed & 31));
           }
         }
@@ -713,7 +711,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         sc_n[SC_SLOT] = 0;
         sc_n[SC_SLOT_E] = 0;
         sc_n[SC_MAXKEY] = 0;
+        scal[SC_NEXT_S] = c1;
       }
+      cp_async_wait_but_one();  // survivors of frame t+1 have landed (visible after B1)
     }
     if (use_bt && !is_chore) {
       // SelectTopK's beam_threshold is relative to the exact best score of the frame
@@ -730,9 +730,11 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     // the cut from warp 0.
     auto chore_between = [&]() {
       const int c3 = (t + 3 < len) ? counts[t + 3] : 0;
-      cp_async_wait_but_one();  // survivors of frame t+1 have landed
-      __syncwarp();
-      if (t + 1 < len) stage_frame(t + 1, c0, c1);
+      if (t + 1 < len) {
+        stage_tables(t + 1, c0, c1, lane, 32);
+        __syncwarp();
+        if (lane == 0) publish_frame(t + 1, c1);
+      }
       c0 = c1; c1 = c2; c2 = c3;
     };
     auto publish_cut = [&](const Cut& c) {
@@ -758,14 +760,21 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         read_cut(cut);
       }
     } else {
+      // large blocks: warp 0 scans, all the others stage the tables of frame t+1 together
+      const int S_next = scal[SC_NEXT_S];
       if (warp == 0) {
         cut = scan_score_histogram(hist, K);
         if (lane == 0) publish_cut(cut);
-      } else if (is_chore) {
-        chore_between();
+      } else if (t + 1 < len) {
+        stage_tables(t + 1, fi.S, S_next, tid - 32, NT - 32);
       }
       __syncthreads();  // B2 (large blocks only)
       read_cut(cut);
+      if (is_chore) {
+        const int c3 = (t + 3 < len) ? counts[t + 3] : 0;
+        if (lane == 0 && t + 1 < len) publish_frame(t + 1, S_next);
+        c0 = c1; c1 = c2; c2 = c3;
+      }
     }
     // new zero of the relative scores: the upper edge of the first non-empty group of bins
     const float best = -(float)(cut.first * kBinsPerLane) * (1.f / kBinsPerNat);
