@@ -1125,10 +1125,12 @@ size_t decode_smem_bytes(int K, int V) {
   }
 }
 
-int decode_block_threads(int K, int V, bool pruning, int top_n) {
-  // one lane per beam entry for the stay candidates, about three extension candidates per
-  // ext lane, one chore warp.  With pruning on, a quarter of a large vocabulary (at least
-  // eight tokens) is assumed to survive a frame.
+int decode_block_threads(int K, int V, bool pruning, int top_n, bool latency_bound) {
+  // One lane per beam entry for the stay candidates, one chore warp, and ext lanes for the
+  // extension candidates: one candidate per lane, counting at most eight survivors per entry,
+  // when every utterance has an SM to itself (the frame chain is all that matters); about
+  // three per lane when blocks share SMs.  With pruning on, a quarter of a large vocabulary
+  // (at least eight tokens) is assumed to survive a frame.
   long long cols = V;
   if (pruning) {
     cols = V / 4;
@@ -1137,7 +1139,8 @@ int decode_block_threads(int K, int V, bool pruning, int top_n) {
   }
   if (top_n > 0 && top_n < cols) cols = top_n;
   const long long stay = ((long long)K + 31) / 32 * 32;
-  long long ext = ((long long)K * cols / 3 + 31) / 32 * 32;
+  long long ext = latency_bound ? (long long)K * (cols < 8 ? cols : 8) : (long long)K * cols / 3;
+  ext = (ext + 31) / 32 * 32;
   if (ext < 32) ext = 32;
   long long nt = stay + ext + 32;
   if (nt > kMaxThreads) nt = kMaxThreads;
@@ -1178,14 +1181,16 @@ cudaError_t decode_prepare(int K, int V) {
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   if (p.B == 0) return cudaSuccess;
-  int nt = p.block_threads > 0 ? p.block_threads : decode_block_threads(p.K, p.V, p.pruning != 0, p.top_n);
-  if (p.block_threads <= 0 && nt > 512 && p.pruning) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int nt = p.block_threads > 0
+               ? p.block_threads
+               : decode_block_threads(p.K, p.V, p.pruning != 0, p.top_n, p.B <= sms);
+  if (p.block_threads <= 0 && nt > 512 && p.pruning && p.B > sms) {
     // more utterances than SMs: two blocks of 512 threads per SM overlap their frame chains
     // better than one block of 1024 (measured on the subword shape, B = 256)
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (p.B > sms) nt = 512;
+    nt = 512;
   }
   nt = (nt + 31) / 32 * 32;
   if (nt < 96) nt = 96;  // a stay warp, an ext warp and the chore warp

@@ -68,7 +68,7 @@ struct DecodeParams {
 };
 
 size_t decode_smem_bytes(int K, int V);
-int decode_block_threads(int K, int V, bool pruning, int top_n);
+int decode_block_threads(int K, int V, bool pruning, int top_n, bool latency_bound);
 cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
 // keeps at most top_n survivors per frame (no-op for top_n <= 0 or >= V)
 cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s);
