@@ -381,7 +381,9 @@ __device__ __forceinline__ void divmod_small(int e, int d, float inv_d, int& q, 
 
 // KMAX / VMAX > 0: the shared-memory arrays are laid out for that beam width and vocabulary
 // whatever K and V are (K <= KMAX, V <= VMAX), so every array offset is a compile-time
-// constant; 0: laid out for the K and V of the call.
+// constant; 0: laid out for the K and V of the call; -1: likewise, for wide beams (a crowded
+// cut bin is split a second time, and the warps are shared out between the two kinds of
+// candidate anew every frame).
 // BT: beam_threshold is on (the exact best score of every frame is tracked).
 template <int MAXT, int KMAX, int VMAX, bool BT>
 __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
@@ -389,6 +391,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
   const int K = p.K, V = p.V, blank = p.blank;
   const int KS = KMAX > 0 ? KMAX : K;  // strides of the per-entry / per-token arrays
+  constexpr bool kWide = KMAX < 0;
   const int VS = VMAX > 0 ? VMAX : V;
   const Lay L = make_layout(KS, VS);
   const int TS = table_size(KS);
@@ -424,12 +427,13 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   int nsw = (K + 31) >> 5;                   // stay warps: one lane per beam entry if possible
   if (nsw > (NW - 1) / 2) nsw = (NW - 1) / 2;
   if (nsw < 1) nsw = 1;
-  const int NS = nsw << 5;                   // stay lanes
-  const int NX = (NW - 1 - nsw) << 5;        // ext lanes
+  // (wide beams move this split every frame, see the frame loop)
+  int NS = nsw << 5;                         // stay lanes
+  int NX = (NW - 1 - nsw) << 5;              // ext lanes
   const bool is_chore = warp == NW - 1;
-  const bool is_stay = warp < nsw;
-  const bool is_ext = !is_chore && !is_stay;
-  const int xl = tid - NS;                   // index among the ext lanes
+  bool is_stay = warp < nsw;
+  bool is_ext = !is_chore && !is_stay;
+  int xl = tid - NS;                         // index among the ext lanes
   const bool warp_scans = NT <= kSmallBlock;
   constexpr bool use_bt = BT;
 
@@ -599,6 +603,20 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     const int Snb = fi.Snb, blank_j = fi.blank_j;
     const int Sdiv = max(Snb, 1);
     const int next = nb * Snb;  // extension candidates of this frame
+    int dq = fi.dq, dj = fi.dj;  // (q, j) step between a lane's successive extension candidates
+    if (kWide) {
+      // Wide beams share the warps out anew every frame, by the counts of the two kinds of
+      // candidate; a stay candidate takes about as long as four extension candidates.
+      const int ws = 4 * nb, wx = next;
+      int n = ((NW - 1) * ws + ws + wx - 1) / (ws + wx);
+      n = max(1, min(n, min((nb + 31) >> 5, NW - 2)));
+      NS = n << 5;
+      NX = (NW - 1 - n) << 5;
+      is_stay = warp < n;
+      is_ext = !is_chore && !is_stay;
+      xl = tid - NS;
+      divmod_small(NX, Sdiv, fi.inv_s, dq, dj);
+    }
 
     // position of the j-th non-blank survivor in the survivor list
     const int blank_at = blank_j >= 0 ? blank_j : 0x7fffffff;
@@ -644,14 +662,14 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     // this lane's extension candidates: e_first, e_first + NX, ... as (q, j) pairs
     int q0 = 0, j0 = 0;
     auto step = [&](int& q, int& j) {
-      q += fi.dq;
-      j += fi.dj;
+      q += dq;
+      j += dj;
       if (j >= Sdiv) { j -= Sdiv; ++q; }
     };
     // (q, j) of this lane's k-th extension candidate
     auto nth = [&](int k, int& q, int& j) {
-      q = q0 + k * fi.dq;
-      j = j0 + k * fi.dj;
+      q = q0 + k * dq;
+      j = j0 + k * dj;
       while (j >= Sdiv) { j -= Sdiv; ++q; }
     };
 
@@ -703,6 +721,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       uint4* dup_n = reinterpret_cast<uint4*>(dup_base + (par ^ 1) * DW);
       uint4* tb_n = reinterpret_cast<uint4*>(tab_n);
       for (int i = lane; i < kFastBins / 4; i += 32) hist_n[i] = zero;
+      if (kWide)
+        for (int i = lane; i < kFastBins / 4; i += 32) reinterpret_cast<uint4*>(rhist)[i] = zero;
       for (int i = lane; i < DW / 4; i += 32) dup_n[i] = zero;
       for (int i = lane; i < TS / 4; i += 32) tb_n[i] = ones;
       if (lane == 0) {
@@ -840,14 +860,55 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       else place_ext(q, ext_token(j1 - 1), key, slot);
     };
 
-    if (take_all || use_list) {
-      // the cut as scores (bin edges): score > f_hi is above the cut bin, score > f_lo is in
-      // it or above.  A score of -inf passes neither.
-      const float f_lo = (cut.thr >= kFastBins - 1) ? neg_inf()
-                                                    : -(float)(cut.thr + 1) * (1.f / kBinsPerNat);
-      const float f_hi = take_all ? f_lo
-                                  : (cut.thr == 0 ? __int_as_float(0x7f800000)
-                                                  : -(float)cut.thr * (1.f / kBinsPerNat));
+    // the cut as scores (bin edges): score > f_hi is above the cut bin, score > f_lo is in it
+    // or above.  A score of -inf passes neither.
+    const float hi_edge = -(float)cut.thr * (1.f / kBinsPerNat);
+    const float f_lo = (cut.thr >= kFastBins - 1) ? neg_inf()
+                                                  : -(float)(cut.thr + 1) * (1.f / kBinsPerNat);
+    const float f_hi = take_all ? f_lo : (cut.thr == 0 ? __int_as_float(0x7f800000) : hi_edge);
+    // A crowded cut bin (wide beams) is split once more, into 256 sub-bins over its quarter
+    // nat, and the cut is located among those.
+    auto sub_bin = [&](float sc) -> int {
+      const int b2 = __float2int_rz((hi_edge - sc) * (kBinsPerNat * (float)kFastBins));
+      return min(kFastBins - 1, max(0, b2));
+    };
+    bool refined = false;
+    int sub_thr = 0, sub_left = 0, sub_count = 0;
+    if (kWide && !take_all && !use_list && cut.thr < kFastBins - 1) {
+      unsigned* const h2 = rhist;  // its first 256 words are cleared every frame by the chore warp
+      if (is_stay) {
+        for (int i = tid; i < nb; i += NS) {
+          const float sc = st_tot[i];
+          if (sc > f_lo && !(sc > f_hi)) atomicAdd(&h2[sub_bin(sc)], 1u);
+        }
+      } else if (is_ext) {
+        int q = q0, j = j0;
+        for (int e = xl; e < next; e += NX) {
+          const float sc = ext_score(hc[q], j);
+          if (sc > f_lo && !(sc > f_hi) && !merged(e)) atomicAdd(&h2[sub_bin(sc)], 1u);
+          step(q, j);
+        }
+      }
+      __syncthreads();
+      const Cut c2 = scan_score_histogram(h2, cut.left);
+      sub_thr = c2.thr; sub_left = c2.left; sub_count = c2.cut_count;
+      refined = c2.total > cut.left;  // always, unless NaN scores upset the counts
+    }
+    const bool take_all2 = refined && sub_count == sub_left;
+    // 2: the candidate takes a beam slot, 1: it is in the (sub-)bin that the cut runs through,
+    // 0: it is out
+    auto klass = [&](float sc) -> int {
+      if (sc > f_hi) return 2;
+      if (!(sc > f_lo)) return 0;
+      if (!kWide || !refined) return 1;
+      const int sb = sub_bin(sc);
+      if (sb < sub_thr || (take_all2 && sb == sub_thr)) return 2;
+      return sb == sub_thr ? 1 : 0;
+    };
+    const int n_listed = refined ? (take_all2 ? 0 : sub_count) : (take_all ? 0 : cut.cut_count);
+    const int n_winners = refined ? sub_left : cut.left;
+
+    if (take_all || use_list || (refined && n_listed <= kListCap)) {
       // P3a: every candidate above the cut bin takes a beam slot and is noted there; stays
       // fill the beam from slot 0 upwards, extensions from the last slot downwards.
       auto list_add = [&](unsigned key, int id) {
@@ -862,7 +923,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         for (int base = 0; base < nb; base += NS) {
           const int i = base + tid;
           const float sc = i < nb ? st_tot[i] : neg_inf();
-          const bool sel = sc > f_hi;
+          const int kl = klass(sc);
+          const bool sel = kl == 2;
           const unsigned m = __ballot_sync(kFull, sel);
           if (m) {
             int at = 0;
@@ -873,16 +935,17 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
               sel_id[at] = i << 16;
             }
           }
-          if (!sel && sc > f_lo) list_add(score_key(sc), i << 16);
+          if (kl == 1) list_add(score_key(sc), i << 16);
         }
       } else if (is_ext) {
         // extensions in the cut bin or above: the lanes of a warp that arrive here together
         // take their places with one atomic
         auto settle = [&](int e, int q, int j, float sc) {
-          if (merged(e)) return;
+          const int kl = klass(sc);
+          if (kl == 0 || merged(e)) return;
           const unsigned key = score_key(sc);
           const int id = (q << 16) | (j + 1);
-          const bool sure = sc > f_hi;
+          const bool sure = kl == 2;
           const unsigned act = __activemask();
           const unsigned ms = __ballot_sync(act, sure);
           const unsigned mine = sure ? ms : (act & ~ms);
@@ -935,16 +998,16 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           const int slot = nbn - 1 - x;
           if (slot >= 0) place_by_id(sel_id[slot], sel_key[slot], slot);
         }
-      } else if (!take_all) {
-        for (int li = lane; li < cut.cut_count; li += 32) {
+      } else {
+        for (int li = lane; li < n_listed; li += 32) {
           const unsigned key = list_key[li];
           const int id = list_id[li];
           int rank = 0;
-          for (int j = 0; j < cut.cut_count; ++j) {
+          for (int j = 0; j < n_listed; ++j) {
             const unsigned kj = list_key[j];
             rank += (kj > key || (kj == key && list_id[j] < id)) ? 1 : 0;
           }
-          if (rank < cut.left) place_by_id(id, key, n_stay + rank);
+          if (rank < n_winners) place_by_id(id, key, n_stay + rank);
         }
       }
     } else {
@@ -1110,11 +1173,12 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
 
 // Layout variants: small beams over a character or a subword vocabulary get compile-time
 // array offsets, everything else the generic kernel.
-enum Variant { kCharBeam64, kSubwordBeam64, kGeneric };
+enum Variant { kCharBeam64, kSubwordBeam64, kGeneric, kWideBeam };
+constexpr int kWideBeamFrom = 257;  // measured: the wide-beam devices pay off from here
 Variant pick_variant(int K, int V) {
   if (K <= 64 && V <= 32) return kCharBeam64;
   if (K <= 64 && V <= 1024) return kSubwordBeam64;
-  return kGeneric;
+  return K >= kWideBeamFrom ? kWideBeam : kGeneric;
 }
 
 size_t decode_smem_bytes(int K, int V) {
@@ -1175,6 +1239,7 @@ cudaError_t decode_prepare(int K, int V) {
   switch (pick_variant(K, V)) {
     case kCharBeam64: return prepare_variant<64, 32>(bytes);
     case kSubwordBeam64: return prepare_variant<64, 1024>(bytes);
+    case kWideBeam: return prepare_variant<-1, 0>(bytes);
     default: return prepare_variant<0, 0>(bytes);
   }
 }
@@ -1199,6 +1264,7 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   switch (pick_variant(p.K, p.V)) {
     case kCharBeam64: launch_variant<64, 32>(p, nt, bytes, s); break;
     case kSubwordBeam64: launch_variant<64, 1024>(p, nt, bytes, s); break;
+    case kWideBeam: launch_variant<-1, 0>(p, nt, bytes, s); break;
     default: launch_variant<0, 0>(p, nt, bytes, s); break;
   }
   return cudaGetLastError();
