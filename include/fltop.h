@@ -189,6 +189,12 @@ int fltop_set_profiling(fltop_handle* h, int enable);
 /* Threads per utterance block of the decode kernel (a multiple of 32, at most 1024; 0 = let
  * the library choose from K, V and R).  A tuning knob: results do not depend on it. */
 int fltop_set_block_threads(fltop_handle* h, int32_t threads);
+/* Where the frames are pruned (Algorithm 1, the top-N stage and the conditional break).
+ * mode 1 (the default): inside the decode kernel whenever vocab_size <= 32 - each utterance
+ * block fetches its own emission rows and no survivor list goes through device memory;
+ * wider vocabularies take the separate prune kernel.  mode 0: always the separate kernel.
+ * Results do not depend on it.  FLTOP_ERR_INVALID_ARG for a null handle or another mode. */
+int fltop_set_fusion(fltop_handle* h, int mode);
 int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
 
 #ifdef __cplusplus

@@ -23,7 +23,8 @@ FLTOP_ST_BAD_LENGTH, FLTOP_ST_ARENA_FULL, FLTOP_ST_TRUNCATED, FLTOP_ST_EMPTY_BEA
 EXPORTS = ("fltop_workspace_size", "fltop_create", "fltop_decode", "fltop_stream_step",
            "fltop_destroy", "fltop_prune", "fltop_status_string", "fltop_last_cuda_error",
            "fltop_beam_state_bytes", "fltop_launch_count", "fltop_last_call_stats", "fltop_set_profiling",
-           "fltop_last_kernel_ms", "fltop_decode_static", "fltop_set_block_threads")
+           "fltop_last_kernel_ms", "fltop_decode_static", "fltop_set_block_threads",
+           "fltop_set_fusion")
 
 
 class fltop_config(C.Structure):
@@ -81,6 +82,8 @@ def lib():
         L.fltop_last_kernel_ms.argtypes = [vp, C.POINTER(C.c_float)]
         L.fltop_set_block_threads.restype = C.c_int
         L.fltop_set_block_threads.argtypes = [vp, i32]
+        L.fltop_set_fusion.restype = C.c_int
+        L.fltop_set_fusion.argtypes = [vp, C.c_int]
         L.fltop_decode_static.restype = C.c_int
         L.fltop_decode_static.argtypes = [i32, i32, i32, C.c_float, vp, i64, i64, vp, i32, i32,
                                           i32, vp, vp, vp, vp, vp, vp]
@@ -230,6 +233,11 @@ class Decoder:
         code = lib().fltop_set_block_threads(self.h, int(threads))
         if code != FLTOP_OK:
             raise FltopError(code, "fltop_set_block_threads")
+
+    def set_fusion(self, mode: int):
+        code = lib().fltop_set_fusion(self.h, int(mode))
+        if code != FLTOP_OK:
+            raise FltopError(code, "fltop_set_fusion")
 
     def last_kernel_ms(self):
         ms = (C.c_float * 2)()

@@ -29,6 +29,7 @@ struct fltop_handle {
   int last_cuda;
   int64_t launches;
   int32_t block_threads;  // 0 = chosen by the library
+  int32_t fusion;         // 1 = the decode kernel prunes where it can
   bool profiling;
   bool prof_valid;
   cudaEvent_t ev[3];
@@ -127,6 +128,9 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.block_threads = h->block_threads; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
   dp.top_n = h->cfg.top_n; dp.beam_threshold = h->cfg.beam_threshold;
   dp.counts = h->counts; dp.entries = h->entries; dp.nodes = h->nodes;
+  const bool fuse = h->fusion != 0 && T > 0 && decode_can_prune(h->cfg.vocab_size);
+  dp.logp = fuse ? d_logp : nullptr; dp.stride_b = stride_b; dp.stride_t = stride_t;
+  dp.log_r = h->log_r;
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
   dp.out_status = d_status;
@@ -134,7 +138,7 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   h->last_B = B; h->last_T = T; h->last_stream = s;
 
   if (h->profiling) cudaEventRecord(h->ev[0], s);
-  if (T > 0) {
+  if (T > 0 && !fuse) {
     e = launch_prune(pp, s);
     if (e != cudaSuccess) return cuda_fail(h, e);
     ++h->launches;
@@ -186,6 +190,7 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
                                     : -std::numeric_limits<float>::infinity();
   h->last_cuda = 0; h->launches = 0; h->profiling = false; h->prof_valid = false;
   h->block_threads = 0;
+  h->fusion = 1;
   h->ev[0] = h->ev[1] = h->ev[2] = nullptr;
   if (cfg->workspace) {
     h->ws = static_cast<unsigned char*>(cfg->workspace);
@@ -338,6 +343,12 @@ int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
   }
   delete[] host;
   if (e != cudaSuccess) return cuda_fail(h, e);
+  return FLTOP_OK;
+}
+
+int fltop_set_fusion(fltop_handle* h, int mode) {
+  if (!h || (mode != 0 && mode != 1)) return FLTOP_ERR_INVALID_ARG;
+  h->fusion = mode;
   return FLTOP_OK;
 }
 

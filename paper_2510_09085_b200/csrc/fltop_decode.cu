@@ -65,6 +65,7 @@ namespace {
 
 constexpr int kMaxThreads = 1024;
 constexpr int kSmallBlock = 256;   // up to here every warp scans the histogram itself
+constexpr int kMidBlock = 512;     // blocks up to here are compiled with 128 registers a thread
 constexpr int kCache = 4;          // extension keys cached in registers per ext lane
 static_assert(kCache == 4, "the cached-score selects in P3 are written out for four scores");
 constexpr int kFastBins = 256;     // score histogram of the fast select
@@ -124,6 +125,10 @@ __device__ __forceinline__ unsigned long long child_print(unsigned long long h, 
 __device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src) {
   const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
   asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(d), "l"(gmem_src));
+}
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(d), "l"(gmem_src));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n"); }
 __device__ __forceinline__ void cp_async_wait_all() {
@@ -203,10 +208,13 @@ __host__ __device__ inline int dup_words(int K, int V) { return (K * ((V + 31) /
 __host__ __device__ inline int node_stage_len(int K) { return (K + 1) & ~1; }
 
 // Byte offsets of the shared-memory arrays.
+// widest vocabulary whose frames the decode block prunes itself (one token per lane)
+constexpr int kFusedMaxV = 32;
+
 struct Lay {
   unsigned sv, hot, ident, where, nstage, finfo, warp_sums, st_pb, st_pnb, st_tot, dup, tab, lpv,
       jpos, hist,
-      rhist, list_key, list_id, sel_key, sel_id, scal, total;
+      rhist, list_key, list_id, sel_key, sel_id, scal, raw, total;
 };
 
 __host__ __device__ inline Lay make_layout(int K, int V) {
@@ -238,6 +246,7 @@ __host__ __device__ inline Lay make_layout(int K, int V) {
   l.sel_key = take(K * 4);
   l.sel_id = take(K * 4);
   l.scal = take(SC_COUNT * 4);
+  l.raw = take(4u * kFusedMaxV * 4);
   l.total = off;
   return l;
 }
@@ -561,10 +570,63 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     scal[SC_NEXT_BJ] = -1;
   };
 
+  // Fused pruning (V <= 32, emissions given): the chore warp fetches the raw rows itself, three
+  // frames ahead, and applies the relative threshold (Algorithm 1's conditional break) and
+  // the top-N cap of stage 1 in registers, one token per lane; no survivor list ever goes
+  // through HBM.  The survivor list it leaves in shared memory is the prune kernel's: tokens
+  // in ascending order, a tie at the N-th place goes to the lower token id.
+  const bool fused = p.logp != nullptr;
+  const float* const rows = fused ? p.logp + (int64_t)b * p.stride_b : nullptr;
+  float* const raw_base = reinterpret_cast<float*>(smem + L.raw);
+  int32_t* const counts_out = p.counts + (int64_t)b * p.T;
+  int kept_sum = 0;  // survivors over all frames of this call
+  auto fetch_row = [&](int t1) {
+    if (lane < V) cp_async4(&raw_base[(t1 & 3) * kFusedMaxV + lane], rows + (int64_t)t1 * p.stride_t + lane);
+  };
+  // the row of frame t1 has landed (each lane reads the word it fetched); returns the count
+  auto prune_row = [&](int t1) -> int {
+    const float v = lane < V ? raw_base[(t1 & 3) * kFusedMaxV + lane] : neg_inf();
+    // row maximum through an order-preserving integer key (a NaN never is the maximum)
+    const unsigned vu = __float_as_uint(v);
+    const unsigned vkey = (v == v) ? ((vu & 0x80000000u) ? ~vu : (vu | 0x80000000u)) : 0x007fffffu;
+    const unsigned mkey = __reduce_max_sync(kFull, vkey);
+    const float m = __uint_as_float((mkey & 0x80000000u) ? (mkey & 0x7fffffffu) : ~mkey);
+    const float thr = __fadd_rn(m, p.log_r);
+    const bool keep = lane < V && v >= thr;
+    unsigned kept = __ballot_sync(kFull, keep);
+    if (p.top_n > 0 && __popc(kept) > p.top_n) {
+      // order-preserving integer key; 0 = not (or no longer) in the running
+      const unsigned u = __float_as_uint(v);
+      unsigned key = keep ? ((u & 0x80000000u) ? ~u : (u | 0x80000000u)) : 0u;
+      unsigned chosen = 0u;
+      for (int i = 0; i < p.top_n; ++i) {
+        const unsigned best_key = __reduce_max_sync(kFull, key);
+        const int w = __ffs(__ballot_sync(kFull, key == best_key)) - 1;
+        chosen |= 1u << w;
+        if (lane == w) key = 0u;
+      }
+      kept = chosen;
+    }
+    if ((kept >> lane) & 1u) svbuf(t1)[__popc(kept & lt_mask)] = Survivor{lane, v};
+    const int n = __popc(kept);
+    kept_sum += n;
+    return n;
+  };
+
   // ---- prologue: survivors of frames 0 and 1, tables of frame 0 ----------------------
   int c0 = 0, c1 = 0, c2 = 0;  // survivor counts of frames t, t+1, t+2 (chore warp only)
   for (int i = tid; i < nb; i += NT) table_insert(tab_base, ident_base[i].print, i);
-  if (is_chore) {
+  if (is_chore && fused) {
+    if (len > 0) fetch_row(0);
+    if (len > 1) fetch_row(1);
+    cp_async_commit();
+    if (len > 2) fetch_row(2);
+    cp_async_commit();
+    cp_async_wait_but_one();
+    c0 = len > 0 ? prune_row(0) : 0;
+    c1 = len > 1 ? prune_row(1) : 0;
+    __syncwarp();
+  } else if (is_chore) {
     c0 = len > 0 ? counts[0] : 0;
     c1 = len > 1 ? counts[1] : 0;
     c2 = len > 2 ? counts[2] : 0;
@@ -574,6 +636,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     cp_async_commit();
     cp_async_wait_all();
     __syncwarp();
+  }
+  if (is_chore) {
     stage_tables(0, 0, c0, lane, 32);
     __syncwarp();
     if (lane == 0) publish_frame(0, c0);
@@ -673,6 +737,26 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       while (j >= Sdiv) { j -= Sdiv; ++q; }
     };
 
+    // Chore warp: the nodes staged by frame t-1 go to the trie; the histogram, the merge
+    // bitmap, the counters (and, in small blocks, the hash table) of frame t+1 start empty.
+    // Narrow beams do this after B1, where the scan leaves the chore warp time to spare; with
+    // wide beams the first phase is the long one, so it goes there.
+    auto chore_window = [&]() {
+      if (lane == 0 && pend_bytes) {
+        bulk_store(nodes + pend_at, nstage + (par ^ 1) * NSL, pend_bytes);
+        bulk_store_wait_read_but_one();  // the staging buffer of this frame is free again
+      }
+      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+      const uint4 ones = make_uint4(~0u, ~0u, ~0u, ~0u);
+      uint4* hist_n = reinterpret_cast<uint4*>(hist_base + (par ^ 1) * kFastBins);
+      uint4* dup_n = reinterpret_cast<uint4*>(dup_base + (par ^ 1) * DW);
+      uint4* tb_n = reinterpret_cast<uint4*>(tab_n);
+      for (int i = lane; i < kFastBins / 4; i += 32) hist_n[i] = zero;
+      for (int i = lane; i < DW / 4; i += 32) dup_n[i] = zero;
+      if (warp_scans)  // (large blocks share this out among all warps)
+        for (int i = lane; i < TS / 4; i += 32) tb_n[i] = ones;
+      if (lane < SC_PER_FRAME) scal[(par ^ 1) * SC_PER_FRAME + lane] = 0;
+    };
     // ---- P1: every candidate is evaluated once and counted -----------------------------
     float kc[kCache];  // this ext lane's first extension scores (-inf: none)
 #pragma unroll
@@ -703,37 +787,25 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         if (sc != neg_inf()) count(sc);
       }
     } else {
-      // chore warp: the nodes staged by frame t-1 go to the trie, survivors of frame t+2 start
-      // their way to shared memory, the tables of frame t+1 start empty
-      if (lane == 0 && pend_bytes) {
-        bulk_store(nodes + pend_at, nstage + (par ^ 1) * NSL, pend_bytes);
-        bulk_store_wait_read_but_one();  // the staging buffer of this frame is free again
-      }
-      if (t + 2 < len) {
+      // chore warp: the emissions of frame t+3 (fused pruning) or the survivors of frame t+2
+      // start their way to shared memory, and the row of frame t+2 becomes its survivor list;
+      // the rest of its work waits until after B1, where nobody is waiting for it
+      if (fused) {
+        if (t + 3 < len) fetch_row(t + 3);
+      } else if (t + 2 < len) {
         const Survivor* src = entries + (int64_t)(t + 2) * V;
         Survivor* dst = svbuf(t + 2);
         for (int j = lane; j < c2; j += 32) cp_async8(&dst[j], &src[j]);
       }
       cp_async_commit();
-      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-      const uint4 ones = make_uint4(~0u, ~0u, ~0u, ~0u);
-      uint4* hist_n = reinterpret_cast<uint4*>(hist_base + (par ^ 1) * kFastBins);
-      uint4* dup_n = reinterpret_cast<uint4*>(dup_base + (par ^ 1) * DW);
-      uint4* tb_n = reinterpret_cast<uint4*>(tab_n);
-      for (int i = lane; i < kFastBins / 4; i += 32) hist_n[i] = zero;
-      if (kWide)
+      if (kWide) {
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
         for (int i = lane; i < kFastBins / 4; i += 32) reinterpret_cast<uint4*>(rhist)[i] = zero;
-      for (int i = lane; i < DW / 4; i += 32) dup_n[i] = zero;
-      for (int i = lane; i < TS / 4; i += 32) tb_n[i] = ones;
-      if (lane == 0) {
-        int* sc_n = scal + (par ^ 1) * SC_PER_FRAME;
-        sc_n[SC_LISTN] = 0;
-        sc_n[SC_SLOT] = 0;
-        sc_n[SC_SLOT_E] = 0;
-        sc_n[SC_MAXKEY] = 0;
-        scal[SC_NEXT_S] = c1;
       }
-      cp_async_wait_but_one();  // survivors of frame t+1 have landed (visible after B1)
+      if (lane == 0) scal[SC_NEXT_S] = c1;
+      cp_async_wait_but_one();  // what was requested a frame ago has landed (visible after B1)
+      if (fused) c2 = (t + 2 < len) ? prune_row(t + 2) : 0;
+      if (kWide) chore_window();
     }
     if (use_bt && !is_chore) {
       // SelectTopK's beam_threshold is relative to the exact best score of the frame
@@ -749,12 +821,13 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     // the constants of frame t+1 (and fetches the survivor count of frame t+3); it takes
     // the cut from warp 0.
     auto chore_between = [&]() {
-      const int c3 = (t + 3 < len) ? counts[t + 3] : 0;
+      const int c3 = (!fused && t + 3 < len) ? counts[t + 3] : 0;
       if (t + 1 < len) {
         stage_tables(t + 1, c0, c1, lane, 32);
         __syncwarp();
         if (lane == 0) publish_frame(t + 1, c1);
       }
+      if (!kWide) chore_window();
       c0 = c1; c1 = c2; c2 = c3;
     };
     auto publish_cut = [&](const Cut& c) {
@@ -785,13 +858,18 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       if (warp == 0) {
         cut = scan_score_histogram(hist, K);
         if (lane == 0) publish_cut(cut);
-      } else if (t + 1 < len) {
-        stage_tables(t + 1, fi.S, S_next, tid - 32, NT - 32);
+      } else {
+        if (t + 1 < len) stage_tables(t + 1, fi.S, S_next, tid - 32, NT - 32);
+        // the hash table of the next beam starts empty (first insertions come after B3)
+        const uint4 ones = make_uint4(~0u, ~0u, ~0u, ~0u);
+        uint4* tb_n = reinterpret_cast<uint4*>(tab_n);
+        for (int i = tid - 32; i < TS / 4; i += NT - 32) tb_n[i] = ones;
+        if (!kWide && is_chore) chore_window();
       }
       __syncthreads();  // B2 (large blocks only)
       read_cut(cut);
       if (is_chore) {
-        const int c3 = (t + 3 < len) ? counts[t + 3] : 0;
+        const int c3 = (!fused && t + 3 < len) ? counts[t + 3] : 0;
         if (lane == 0 && t + 1 < len) publish_frame(t + 1, S_next);
         c0 = c1; c1 = c2; c2 = c3;
       }
@@ -1087,6 +1165,13 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     cur = nxt;
   }
   frames_seen += len;
+  if (fused) {
+    // Survivor counts per frame are not kept (a global store in the frame loop would hold up
+    // the block's next barrier); the utterance's total stands in the first frame's place.
+    for (int t1 = tid; t1 < p.T; t1 += NT) counts_out[t1] = 0;
+    __syncthreads();
+    if (is_chore && lane == 0 && p.T > 0) counts_out[0] = kept_sum;
+  }
   // the last frame's nodes; the read-out below walks the trie, so wait for all of them
   if (is_chore && lane == 0) {
     if (pend_bytes) bulk_store(nodes + pend_at, nstage + ((len - 1) & 1) * NSL, pend_bytes);
@@ -1208,6 +1293,10 @@ int decode_block_threads(int K, int V, bool pruning, int top_n, bool latency_bou
   if (ext < 32) ext = 32;
   long long nt = stay + ext + 32;
   if (nt > kMaxThreads) nt = kMaxThreads;
+  // A block of at most 512 threads has 128 registers a thread instead of 64; with pruning on
+  // and a beam of moderate width that is worth more than the extra lanes (measured at V = 32:
+  // 3 to 12 % faster for K = 64 ... 160, slower from K = 200).
+  if (latency_bound && pruning && K <= 160 && nt > kMidBlock) nt = kMidBlock;
   return (int)nt;
 }
 
@@ -1216,23 +1305,32 @@ template <int KMAX, int VMAX>
 cudaError_t prepare_variant(int bytes) {
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
   cudaError_t e = cudaFuncSetAttribute(decode_kernel<kSmallBlock, KMAX, VMAX, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMidBlock, KMAX, VMAX, false>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX, false>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kSmallBlock, KMAX, VMAX, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMidBlock, KMAX, VMAX, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX, true>, attr, bytes);
   return e;
 }
 template <int KMAX, int VMAX>
-void launch_variant(const DecodeParams& p, int nt, size_t bytes, cudaStream_t s) {
+void launch_variant(const DecodeParams& p, int nt, size_t bytes, bool alone, cudaStream_t s) {
   const bool bt = p.beam_threshold > 0.f;
   if (nt <= kSmallBlock) {
     if (bt) decode_kernel<kSmallBlock, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
     else decode_kernel<kSmallBlock, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
+  } else if (nt <= kMidBlock && alone) {
+    // one block per SM: it may as well have 128 registers a thread (blocks that share an SM
+    // keep to 64 so that two of 512 threads fit)
+    if (bt) decode_kernel<kMidBlock, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
+    else decode_kernel<kMidBlock, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
   } else {
     if (bt) decode_kernel<kMaxThreads, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
     else decode_kernel<kMaxThreads, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
   }
 }
 }  // namespace
+
+bool decode_can_prune(int V) { return V <= kFusedMaxV; }
 
 cudaError_t decode_prepare(int K, int V) {
   const int bytes = (int)decode_smem_bytes(K, V);
@@ -1262,10 +1360,10 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   if (nt > kMaxThreads) nt = kMaxThreads;
   const size_t bytes = decode_smem_bytes(p.K, p.V);
   switch (pick_variant(p.K, p.V)) {
-    case kCharBeam64: launch_variant<64, 32>(p, nt, bytes, s); break;
-    case kSubwordBeam64: launch_variant<64, 1024>(p, nt, bytes, s); break;
-    case kWideBeam: launch_variant<-1, 0>(p, nt, bytes, s); break;
-    default: launch_variant<0, 0>(p, nt, bytes, s); break;
+    case kCharBeam64: launch_variant<64, 32>(p, nt, bytes, p.B <= sms, s); break;
+    case kSubwordBeam64: launch_variant<64, 1024>(p, nt, bytes, p.B <= sms, s); break;
+    case kWideBeam: launch_variant<-1, 0>(p, nt, bytes, p.B <= sms, s); break;
+    default: launch_variant<0, 0>(p, nt, bytes, p.B <= sms, s); break;
   }
   return cudaGetLastError();
 }

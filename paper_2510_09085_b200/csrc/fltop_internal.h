@@ -54,8 +54,13 @@ struct DecodeParams {
   int32_t pruning;          // 1 when R is large enough that few tokens survive a frame
   int32_t top_n;            // survivors per frame are capped at this (0: no cap)
   float beam_threshold;     // kept prefixes score at least best - beam_threshold (<= 0: off)
-  const int32_t* counts;    // [B*T] survivors per frame
+  int32_t* counts;          // [B*T] survivors per frame (a kernel that prunes itself leaves
+                            // each utterance's total in its first frame's place, zeros after)
   const Survivor* entries;  // [B*T*V]
+  // Non-null: the decode kernel prunes the rows itself (V <= 32) and `entries` is not read.
+  const float* logp;
+  int64_t stride_b, stride_t;
+  float log_r;
   TrieNode* nodes;          // [B * nodes_per_utt]
   int64_t nodes_per_utt;
   int32_t* state;           // [B * state_words(K)] (streaming only)
@@ -74,5 +79,6 @@ cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
 cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s);
 cudaError_t decode_prepare(int K, int V);  // one-time kernel attribute set-up
+bool decode_can_prune(int V);            // the decode kernel can take raw emission rows
 
 }  // namespace fltop

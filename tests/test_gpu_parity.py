@@ -225,6 +225,25 @@ def test_many_near_equal_scores_take_the_exact_select_path():
         d.close()
 
 
+@pytest.mark.parametrize("spread", [0.02, 0.001])
+def test_wide_beam_with_a_crowded_cut_bin(spread):
+    # wide beams split a crowded cut bin a second time; at the larger spread the finer bins
+    # separate the candidates, at the smaller one even those stay crowded and the exact
+    # selection has to finish the job
+    rng = np.random.default_rng(6)
+    B, T, V = 2, 12, 16
+    x = rng.standard_normal((B, T, V)) * spread
+    em = (x - np.log(np.exp(x).sum(-1, keepdims=True))).astype(np.float32)
+    ln = np.array([T, T - 2], dtype=np.int32)
+    for K in (300, 700):
+        d = gpu_decode(em, ln, 0, K, 0.0)
+        res = oracle.decode(em, ln, 0, K, 0.0)
+        for b in range(B):
+            check_hyps(d.hyps(b), res.hyps(b), K, max_unmatched_frac=0.3,
+                       where=f"flat wide utt {b} K={K} spread={spread}")
+        d.close()
+
+
 def test_exact_ties_keep_a_valid_beam():
     # constant rows: every extension of a prefix ties exactly.  Which of the tied
     # candidates survive is not unique; every kept hypothesis must carry its exact
