@@ -189,7 +189,7 @@ enum {
   SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_MAXKEY, SC_PER_FRAME,
   // single copies
   SC_THR = 2 * SC_PER_FRAME, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_TOTAL, SC_FIRST, SC_STATUS,
-  SC_CREATED, SC_DEAD, SC_NLIVE, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL,
+  SC_CREATED, SC_DEAD, SC_NLIVE, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL, SC_KEPT,
   // exact fallback select
   SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_NBEAM_NEXT, SC_COUNT
 };
@@ -225,6 +225,7 @@ __host__ __device__ inline Lay make_layout(int K, int V) {
     off += (bytes + 15u) & ~15u;
     return at;
   };
+  l.raw = take(4u * kFusedMaxV * 4);  // first: its address needs no offset
   l.sv = take(4u * V * 8);
   l.hot = take(2u * K * 16);
   l.ident = take(2u * K * 16);
@@ -246,7 +247,6 @@ __host__ __device__ inline Lay make_layout(int K, int V) {
   l.sel_key = take(K * 4);
   l.sel_id = take(K * 4);
   l.scal = take(SC_COUNT * 4);
-  l.raw = take(4u * kFusedMaxV * 4);
   l.total = off;
   return l;
 }
@@ -575,17 +575,19 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   // the top-N cap of stage 1 in registers, one token per lane; no survivor list ever goes
   // through HBM.  The survivor list it leaves in shared memory is the prune kernel's: tokens
   // in ascending order, a tie at the N-th place goes to the lower token id.
-  const bool fused = p.logp != nullptr;
-  const float* const rows = fused ? p.logp + (int64_t)b * p.stride_b : nullptr;
-  float* const raw_base = reinterpret_cast<float*>(smem + L.raw);
-  int32_t* const counts_out = p.counts + (int64_t)b * p.T;
-  int kept_sum = 0;  // survivors over all frames of this call
+  // (Nothing of this is kept in registers across the frame loop: the large blocks have 64 a
+  // thread, and every thread would pay for what only the chore warp uses.)
+  auto fused = [&]() -> bool { return p.logp != nullptr; };
+  auto raw_row = [&](int t1) -> float* {
+    return reinterpret_cast<float*>(smem) + (t1 & 3) * kFusedMaxV;
+  };
   auto fetch_row = [&](int t1) {
-    if (lane < V) cp_async4(&raw_base[(t1 & 3) * kFusedMaxV + lane], rows + (int64_t)t1 * p.stride_t + lane);
+    if (lane < V)
+      cp_async4(raw_row(t1) + lane, p.logp + (int64_t)b * p.stride_b + (int64_t)t1 * p.stride_t + lane);
   };
   // the row of frame t1 has landed (each lane reads the word it fetched); returns the count
   auto prune_row = [&](int t1) -> int {
-    const float v = lane < V ? raw_base[(t1 & 3) * kFusedMaxV + lane] : neg_inf();
+    const float v = lane < V ? raw_row(t1)[lane] : neg_inf();
     // row maximum through an order-preserving integer key (a NaN never is the maximum)
     const unsigned vu = __float_as_uint(v);
     const unsigned vkey = (v == v) ? ((vu & 0x80000000u) ? ~vu : (vu | 0x80000000u)) : 0x007fffffu;
@@ -609,14 +611,14 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     }
     if ((kept >> lane) & 1u) svbuf(t1)[__popc(kept & lt_mask)] = Survivor{lane, v};
     const int n = __popc(kept);
-    kept_sum += n;
+    if (lane == 0) scal[SC_KEPT] += n;  // survivors over all frames of this call
     return n;
   };
 
   // ---- prologue: survivors of frames 0 and 1, tables of frame 0 ----------------------
   int c0 = 0, c1 = 0, c2 = 0;  // survivor counts of frames t, t+1, t+2 (chore warp only)
   for (int i = tid; i < nb; i += NT) table_insert(tab_base, ident_base[i].print, i);
-  if (is_chore && fused) {
+  if (is_chore && fused()) {
     if (len > 0) fetch_row(0);
     if (len > 1) fetch_row(1);
     cp_async_commit();
@@ -790,7 +792,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       // chore warp: the emissions of frame t+3 (fused pruning) or the survivors of frame t+2
       // start their way to shared memory, and the row of frame t+2 becomes its survivor list;
       // the rest of its work waits until after B1, where nobody is waiting for it
-      if (fused) {
+      if (fused()) {
         if (t + 3 < len) fetch_row(t + 3);
       } else if (t + 2 < len) {
         const Survivor* src = entries + (int64_t)(t + 2) * V;
@@ -804,7 +806,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       }
       if (lane == 0) scal[SC_NEXT_S] = c1;
       cp_async_wait_but_one();  // what was requested a frame ago has landed (visible after B1)
-      if (fused) c2 = (t + 2 < len) ? prune_row(t + 2) : 0;
+      if (fused()) c2 = (t + 2 < len) ? prune_row(t + 2) : 0;
       if (kWide) chore_window();
     }
     if (use_bt && !is_chore) {
@@ -821,7 +823,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     // the constants of frame t+1 (and fetches the survivor count of frame t+3); it takes
     // the cut from warp 0.
     auto chore_between = [&]() {
-      const int c3 = (!fused && t + 3 < len) ? counts[t + 3] : 0;
+      const int c3 = (!fused() && t + 3 < len) ? counts[t + 3] : 0;
       if (t + 1 < len) {
         stage_tables(t + 1, c0, c1, lane, 32);
         __syncwarp();
@@ -869,7 +871,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       __syncthreads();  // B2 (large blocks only)
       read_cut(cut);
       if (is_chore) {
-        const int c3 = (!fused && t + 3 < len) ? counts[t + 3] : 0;
+        const int c3 = (!fused() && t + 3 < len) ? counts[t + 3] : 0;
         if (lane == 0 && t + 1 < len) publish_frame(t + 1, S_next);
         c0 = c1; c1 = c2; c2 = c3;
       }
@@ -1165,12 +1167,13 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     cur = nxt;
   }
   frames_seen += len;
-  if (fused) {
+  if (fused()) {
     // Survivor counts per frame are not kept (a global store in the frame loop would hold up
     // the block's next barrier); the utterance's total stands in the first frame's place.
+    int32_t* const counts_out = p.counts + (int64_t)b * p.T;
     for (int t1 = tid; t1 < p.T; t1 += NT) counts_out[t1] = 0;
     __syncthreads();
-    if (is_chore && lane == 0 && p.T > 0) counts_out[0] = kept_sum;
+    if (tid == 0 && p.T > 0) counts_out[0] = scal[SC_KEPT];
   }
   // the last frame's nodes; the read-out below walks the trie, so wait for all of them
   if (is_chore && lane == 0) {
