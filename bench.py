@@ -34,7 +34,22 @@ L2_FLUSH_BYTES = 256 << 20
 NODE_BYTES, SURVIVOR_BYTES = 8, 8
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch on the default workload
 # (profiles/decode_kernel_wav2vec2_B64_K50_full.txt); None whenever the kernel has changed since
-DECODE_DRAM_BYTES = 9.31e6
+DECODE_DRAM_BYTES = 7.40e6
+
+
+def _algorithmic_bytes(V, st, out_bytes, fused):
+    """(prune kernel, decode kernel) HBM bytes that one call has to move.
+
+    Two kernels: the prune kernel reads every emission row and writes a count and the survivor
+    list per frame, the decode kernel reads those back.  One kernel (it prunes its own rows):
+    the emission rows are the decode kernel's input and no survivor list exists.  Either way
+    the decode kernel writes one block of 8-byte trie records per frame (one record per beam
+    slot, rounded up to an even count) and the hypotheses at the end."""
+    trie = NODE_BYTES * (st["live_hypotheses_sum"] + st["frames"])
+    if fused:
+        return 0, st["frames"] * 4 * V + trie + out_bytes
+    prune = st["frames"] * (4 * V + 4) + st["survivors"] * SURVIVOR_BYTES
+    return prune, st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES + trie + out_bytes
 
 
 def _peaks():
@@ -247,16 +262,11 @@ def run_ours(args):
 
     def kernel_bytes(dec, st):
         """Algorithmic HBM bytes of one launch of each kernel (inputs of this rank)."""
-        n_hyp = int(dec.nhyp.sum())
-        out_bytes = 4 * int(dec.lens.sum()) + 8 * n_hyp + 8 * B
-        prune = st["frames"] * (4 * V + 4) + st["survivors"] * SURVIVOR_BYTES
-        # survivor lists read back, one block of 8-byte trie records per frame (one record
-        # per beam slot, rounded up to an even count), the hypotheses written at the end
-        trie = NODE_BYTES * (st["live_hypotheses_sum"] + st["frames"])
-        decode = st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES + trie + out_bytes
-        return prune, decode
+        out_bytes = 4 * int(dec.lens.sum()) + 8 * int(dec.nhyp.sum()) + 8 * B
+        return _algorithmic_bytes(V, st, out_bytes, fused=(launches_per_step == 1))
 
     peak, peak_kind = _peaks()
+    launches_per_step = launches // max(1, args.steps)
     pb, db = kernel_bytes(dec_p, stats_p)
     pb0, db0 = kernel_bytes(dec_0, stats_0)
     dk_ms = statistics.mean(decode_p)
@@ -319,7 +329,9 @@ def run_ours(args):
             "mean_live_hypotheses": stats_p["live_hypotheses_sum"] / max(1, stats_p["frames"]),
             "trie_nodes_created": stats_p["trie_nodes_created"],
             "hbm_frac_step": (pb + db) / (t_p * 1e-3) / 1e9 / peak,
-            "prune_kernel_gbs": pb / (statistics.mean(prune_p) * 1e-3) / 1e9,
+            "prune_kernel_gbs": (pb / (statistics.mean(prune_p) * 1e-3) / 1e9
+                                 if statistics.mean(prune_p) > 0 else None),
+            "pruning": "inside the decode kernel" if launches_per_step == 1 else "separate kernel",
             "beam_state_bytes": dec_p.beam_state_bytes,
             "step_ms_min": min(ms_p), "step_ms_median": statistics.median(ms_p),
         },
@@ -378,10 +390,8 @@ def run_report(args):
         st = dec.last_call_stats()
         assert int((dec.status != 0).sum()) == 0
         frames = int(wl.lengths.sum())
-        pbytes = st["frames"] * (4 * V + 4) + st["survivors"] * SURVIVOR_BYTES
-        dbytes = (st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES
-                  + NODE_BYTES * (st["live_hypotheses_sum"] + st["frames"])
-                  + 4 * int(dec.lens.sum()) + 8 * int(dec.nhyp.sum()) + 8 * B)
+        pbytes, dbytes = _algorithmic_bytes(
+            V, st, 4 * int(dec.lens.sum()) + 8 * int(dec.nhyp.sum()) + 8 * B, fused=(pk == 0.0))
         agree = None
         if top1_ref is not None:
             agree = sum(dec.hyps(b)[0][0] == top1_ref[b] for b in range(B)) / B
@@ -468,7 +478,8 @@ def run_report(args):
             ag = "" if w["top1_agree"] is None else f"{100 * w['top1_agree']:.1f} %"
             f.write(f"| {w['workload']} | {w['K']} | {w['r']:g} | {w['frames_per_s']:.3g} | "
                     f"{w['utt_per_s']:.3g} | {w['ms']:.3f} | {100 * w['hbm_frac_step']:.3f} % | "
-                    f"{w['prune_gbs']:.0f} | {w['ns_per_frame_step']:.0f} | "
+                    f"{(format(w['prune_gbs'], '.0f') if w['prune_gbs'] else 'in decode')} | "
+                    f"{w['ns_per_frame_step']:.0f} | "
                     f"{w['beam_state_bytes'] / 1e6:.1f} | {w['mean_survivors']:.2f} | "
                     f"{w['mean_live']:.1f} | {ag} |\n")
         f.write(f"\nStreaming (cfg 4, K={K}, r={r:g}, 1024 streams x 100 chunks of 16 frames): "

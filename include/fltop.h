@@ -184,7 +184,8 @@ int64_t fltop_launch_count(const fltop_handle* h);
 int fltop_last_call_stats(fltop_handle* h, int64_t* out);
 /* With profiling enabled every call brackets its kernels with CUDA events on the caller's
  * stream.  fltop_last_kernel_ms synchronises on those events and returns the device time
- * of the most recent call's {prune, decode} kernels in out_ms[0..1] (milliseconds). */
+ * of the most recent call's {prune, decode} kernels in out_ms[0..1] (milliseconds); the
+ * first is 0 when the decode kernel pruned the frames itself (see fltop_set_fusion). */
 int fltop_set_profiling(fltop_handle* h, int enable);
 /* Threads per utterance block of the decode kernel (a multiple of 32, at most 1024; 0 = let
  * the library choose from K, V and R).  A tuning knob: results do not depend on it. */

@@ -22,6 +22,7 @@ struct fltop_handle {
   int32_t* state;
   int32_t* stats;
   int32_t last_B, last_T;
+  bool last_fused;        // the most recent call pruned inside the decode kernel
   cudaStream_t last_stream;
   int64_t frame_cap;      // frames per utterance the survivor buffers hold
   int64_t nodes_per_utt;
@@ -135,7 +136,7 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
   dp.out_status = d_status;
   dp.stats = h->stats;
-  h->last_B = B; h->last_T = T; h->last_stream = s;
+  h->last_B = B; h->last_T = T; h->last_stream = s; h->last_fused = fuse;
 
   if (h->profiling) cudaEventRecord(h->ev[0], s);
   if (T > 0 && !fuse) {
@@ -212,7 +213,7 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   h->nodes = reinterpret_cast<TrieNode*>(h->ws + l.nodes);
   h->state = cfg->max_chunk_frames > 0 ? reinterpret_cast<int32_t*>(h->ws + l.state) : nullptr;
   h->stats = reinterpret_cast<int32_t*>(h->ws + l.stats);
-  h->last_B = 0; h->last_T = 0; h->last_stream = nullptr;
+  h->last_B = 0; h->last_T = 0; h->last_stream = nullptr; h->last_fused = false;
   h->frame_cap = l.frame_cap;
   h->nodes_per_utt = l.nodes_per_utt;
   h->beam_state_bytes = l.beam_state;
@@ -378,6 +379,7 @@ int fltop_last_kernel_ms(fltop_handle* h, float* out_ms) {
   if (e == cudaSuccess) e = cudaEventElapsedTime(&out_ms[0], h->ev[0], h->ev[1]);
   if (e == cudaSuccess) e = cudaEventElapsedTime(&out_ms[1], h->ev[1], h->ev[2]);
   if (e != cudaSuccess) return cuda_fail(h, e);
+  if (h->last_fused) out_ms[0] = 0.f;  // no prune kernel ran
   return FLTOP_OK;
 }
 
