@@ -111,6 +111,33 @@ int fltop_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t
                  int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
                  void* cuda_stream);
 
+/* fltop_decode for callers whose emissions and results live in HOST memory (Algorithm 1 is
+ * stated on host arrays; this is the same procedure with the transfers done by the library).
+ * fltop_enable_host_io allocates, once, what that takes: device copies of the inputs and
+ * outputs ([max_batch, max_frames, V] float32 + [max_batch, K, L] int32 + small arrays), a few
+ * KB of pinned host memory, sixteen streams.  FLTOP_ERR_STATE on a streaming handle,
+ * FLTOP_ERR_OOM / FLTOP_ERR_CUDA if an allocation fails (the handle stays usable for the
+ * device-pointer calls); calling it again is a no-op. */
+int fltop_enable_host_io(fltop_handle* h);
+
+/* Arguments as in fltop_decode, but every h_* pointer is HOST memory (pinned memory lets the
+ * copies run asynchronously; pageable memory works, slower).  The batch is cut into groups of
+ * utterances, longest first; each group's frames are copied (only the h_lengths[b] valid frames
+ * of an utterance), decoded and read back on streams of the handle, so that all transfers but
+ * the first group's overlap with decoding.  Only existing tokens are copied back:
+ * h_tokens[b,k,0:len] for k < nhyp is written, everything else in h_tokens is left untouched;
+ * h_lens, h_scores, h_nhyp and (if not NULL) h_status are written in full.
+ * The work is ordered after what `cuda_stream` held at the call and `cuda_stream` waits for
+ * it; unlike the device-pointer calls this one RETURNS ONLY WHEN THE OUTPUTS ARE IN HOST
+ * MEMORY.  Results are those of fltop_decode, bit for bit.  FLTOP_ERR_STATE unless
+ * fltop_enable_host_io succeeded on this handle. */
+int fltop_decode_host(fltop_handle* h, const float* h_logp, int64_t stride_b, int64_t stride_t,
+                      const int32_t* h_lengths, int32_t B, int32_t T, int32_t* h_tokens,
+                      int32_t* h_lens, float* h_scores, int32_t* h_nhyp, int32_t* h_status,
+                      void* cuda_stream);
+/* Bytes the most recent fltop_decode_host moved: out[0] host to device, out[1] device to host. */
+int fltop_last_host_io_bytes(const fltop_handle* h, int64_t* out);
+
 /* Algorithm 1 consumed chunk by chunk: the frame loop of S concurrent streams advances by
  * up to C frames; the beam of every stream is kept in the handle between calls.
  *   d_chunk      [S,C,V] float32, contiguous.

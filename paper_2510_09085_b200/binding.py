@@ -24,7 +24,8 @@ EXPORTS = ("fltop_workspace_size", "fltop_create", "fltop_decode", "fltop_stream
            "fltop_destroy", "fltop_prune", "fltop_status_string", "fltop_last_cuda_error",
            "fltop_beam_state_bytes", "fltop_launch_count", "fltop_last_call_stats", "fltop_set_profiling",
            "fltop_last_kernel_ms", "fltop_decode_static", "fltop_set_block_threads",
-           "fltop_set_fusion")
+           "fltop_set_fusion", "fltop_enable_host_io", "fltop_decode_host",
+           "fltop_last_host_io_bytes")
 
 
 class fltop_config(C.Structure):
@@ -84,6 +85,12 @@ def lib():
         L.fltop_set_block_threads.argtypes = [vp, i32]
         L.fltop_set_fusion.restype = C.c_int
         L.fltop_set_fusion.argtypes = [vp, C.c_int]
+        L.fltop_enable_host_io.restype = C.c_int
+        L.fltop_enable_host_io.argtypes = [vp]
+        L.fltop_decode_host.restype = C.c_int
+        L.fltop_decode_host.argtypes = [vp, vp, i64, i64, vp, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.fltop_last_host_io_bytes.restype = C.c_int
+        L.fltop_last_host_io_bytes.argtypes = [vp, C.POINTER(C.c_int64)]
         L.fltop_decode_static.restype = C.c_int
         L.fltop_decode_static.argtypes = [i32, i32, i32, C.c_float, vp, i64, i64, vp, i32, i32,
                                           i32, vp, vp, vp, vp, vp, vp]
@@ -191,6 +198,48 @@ class Decoder:
         if code != FLTOP_OK:
             raise FltopError(code, "fltop_decode")
         return self
+
+    # --- batch, host buffers -------------------------------------------------------
+    def enable_host_io(self, pin: bool = True):
+        """Allocates the library's staging and the host output tensors (pinned unless pin=False)."""
+        code = lib().fltop_enable_host_io(self.h)
+        if code != FLTOP_OK:
+            raise FltopError(code, "fltop_enable_host_io")
+        mk = (lambda t: t.pin_memory()) if pin else (lambda t: t)
+        self.h_tokens = mk(torch.zeros(self.tokens.shape, dtype=torch.int32))
+        self.h_lens = mk(torch.zeros(self.lens.shape, dtype=torch.int32))
+        self.h_scores = mk(torch.zeros(self.scores.shape, dtype=torch.float32))
+        self.h_nhyp = mk(torch.zeros(self.nhyp.shape, dtype=torch.int32))
+        self.h_status = mk(torch.zeros(self.status.shape, dtype=torch.int32))
+
+    def decode_host(self, logp: torch.Tensor, lengths: torch.Tensor, stream=None):
+        """logp [B,T,V] float32 and lengths [B] int32 in HOST memory; the results are in the
+        host tensors h_tokens / h_lens / h_scores / h_nhyp / h_status when this returns."""
+        assert not logp.is_cuda and logp.dtype == torch.float32 and logp.stride(2) == 1
+        assert not lengths.is_cuda and lengths.dtype == torch.int32 and lengths.is_contiguous()
+        B, T, _ = logp.shape
+        code = lib().fltop_decode_host(self.h, _p(logp), logp.stride(0), logp.stride(1),
+                                       _p(lengths), B, T, _p(self.h_tokens), _p(self.h_lens),
+                                       _p(self.h_scores), _p(self.h_nhyp), _p(self.h_status),
+                                       _stream_ptr(stream))
+        if code != FLTOP_OK:
+            raise FltopError(code, "fltop_decode_host")
+        return self
+
+    def host_io_bytes(self):
+        """(host-to-device, device-to-host) bytes of the most recent decode_host."""
+        out = (C.c_int64 * 2)()
+        code = lib().fltop_last_host_io_bytes(self.h, out)
+        if code != FLTOP_OK:
+            raise FltopError(code, "fltop_last_host_io_bytes")
+        return int(out[0]), int(out[1])
+
+    def host_hyps(self, b: int):
+        """[(token tuple, score)] of utterance b from the host outputs of decode_host."""
+        n = int(self.h_nhyp[b])
+        lens = self.h_lens[b, :n].tolist()
+        sc = self.h_scores[b, :n].tolist()
+        return [(tuple(self.h_tokens[b, k, : lens[k]].tolist()), sc[k]) for k in range(n)]
 
     # --- streaming -----------------------------------------------------------------
     def stream_step(self, chunk: torch.Tensor, chunk_lens: torch.Tensor, flags=None,

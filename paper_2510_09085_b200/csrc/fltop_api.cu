@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/fltop.h: argument validation,
 // workspace carve-up and kernel launches on the caller's stream.
+#include <algorithm>
 #include <cmath>
 #include <limits>
 #include <new>
@@ -9,8 +10,35 @@
 
 using namespace fltop;
 
+namespace {
+constexpr int kIoMaxGroups = 16;
+constexpr int kIoStreams = kIoMaxGroups;  // a stream per group: the groups' kernels run side by side
+constexpr int kIoGroupSize = 8;  // utterances per group (more when B > 8 * kIoMaxGroups)
+
+// Staging of fltop_decode_host: device copies of the inputs and outputs, pinned host mirrors of
+// the small outputs, the streams and events of the copy / decode pipeline.
+struct HostIo {
+  bool ready = false;
+  unsigned char* dev = nullptr;      // one device allocation
+  unsigned char* pinned = nullptr;   // one pinned host allocation
+  float* d_logp = nullptr;           // [max_batch, max_frames, V]
+  int32_t* d_lengths = nullptr;      // [max_batch]
+  int32_t* d_tokens = nullptr;       // [max_batch, K, L]
+  // lens [n,K], scores [n,K], nhyp [n], status [n] of a group of n utterances lie back to back
+  // (2K + 2 words per utterance), so that one copy brings a group's small outputs home
+  int32_t* d_small = nullptr;        // [max_batch * (2K + 2)]
+  int32_t* p_small = nullptr;        // pinned host mirror
+  int32_t* p_lengths = nullptr;      // pinned, [max_batch], in slot order
+  int32_t* order = nullptr;          // [max_batch] pageable host scratch
+  cudaStream_t stream[kIoStreams] = {};
+  cudaEvent_t begin = nullptr, end[kIoStreams] = {}, done[kIoMaxGroups] = {};
+  int64_t h2d_bytes = 0, d2h_bytes = 0;  // of the most recent call
+};
+}  // namespace
+
 struct fltop_handle {
   fltop_config cfg;
+  HostIo io;
   float log_r;
   bool owns_workspace;
   unsigned char* ws;
@@ -110,7 +138,10 @@ struct DeviceGuard {
 int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
                const int32_t* d_lengths, const uint8_t* d_flags, int32_t B, int32_t T,
                bool streaming, int32_t* d_tokens, int32_t* d_lens, float* d_scores,
-               int32_t* d_nhyp, int32_t* d_status, cudaStream_t s) {
+               int32_t* d_nhyp, int32_t* d_status, cudaStream_t s, int32_t slot0 = 0,
+               int32_t co_resident = 0) {
+  // slot0: first of the handle's per-utterance scratch slots this launch uses (a batch that is
+  // decoded group by group gives every group its own range of slots)
   DeviceGuard g;
   cudaError_t e = g.enter(h->cfg.device);
   if (e != cudaSuccess) return cuda_fail(h, e);
@@ -120,25 +151,29 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   PruneParams pp;
   pp.logp = d_logp; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
-  pp.counts = h->counts; pp.entries = h->entries;
+  pp.counts = h->counts + (int64_t)slot0 * T;
+  pp.entries = h->entries + (int64_t)slot0 * T * h->cfg.vocab_size;
 
   DecodeParams dp;
   dp.lengths = d_lengths; dp.flags = d_flags; dp.B = B; dp.T = T; dp.V = h->cfg.vocab_size;
   dp.K = h->cfg.beam_width; dp.blank = h->cfg.blank_id; dp.L = h->cfg.max_out_len;
   dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
-  dp.block_threads = h->block_threads; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
+  dp.block_threads = h->block_threads; dp.co_resident = co_resident; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
   dp.top_n = h->cfg.top_n; dp.beam_threshold = h->cfg.beam_threshold;
-  dp.counts = h->counts; dp.entries = h->entries; dp.nodes = h->nodes;
+  dp.counts = pp.counts; dp.entries = pp.entries;
+  dp.nodes = h->nodes + (int64_t)slot0 * h->nodes_per_utt;
   const bool fuse = h->fusion != 0 && T > 0 && decode_can_prune(h->cfg.vocab_size);
   dp.logp = fuse ? d_logp : nullptr; dp.stride_b = stride_b; dp.stride_t = stride_t;
   dp.log_r = h->log_r;
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
   dp.out_status = d_status;
-  dp.stats = h->stats;
-  h->last_B = B; h->last_T = T; h->last_stream = s; h->last_fused = fuse;
+  dp.stats = h->stats + (int64_t)slot0 * 4;
+  if (slot0 == 0) { h->last_B = B; h->last_T = T; h->last_stream = s; h->last_fused = fuse; }
 
-  if (h->profiling) cudaEventRecord(h->ev[0], s);
+  // (a batch decoded group by group on several streams is not timed kernel by kernel)
+  const bool timed = h->profiling && co_resident == 0;
+  if (timed) cudaEventRecord(h->ev[0], s);
   if (T > 0 && !fuse) {
     e = launch_prune(pp, s);
     if (e != cudaSuccess) return cuda_fail(h, e);
@@ -149,20 +184,232 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
       ++h->launches;
     }
   }
-  if (h->profiling) cudaEventRecord(h->ev[1], s);
+  if (timed) cudaEventRecord(h->ev[1], s);
   e = launch_decode(dp, s);
   if (e != cudaSuccess) return cuda_fail(h, e);
   ++h->launches;
-  if (h->profiling) {
+  if (timed) {
     cudaEventRecord(h->ev[2], s);
     h->prof_valid = true;
   }
   return FLTOP_OK;
 }
 
+void host_io_release(HostIo& io) {
+  for (int i = 0; i < kIoStreams; ++i) {
+    if (io.stream[i]) cudaStreamDestroy(io.stream[i]);
+    if (io.end[i]) cudaEventDestroy(io.end[i]);
+  }
+  for (int i = 0; i < kIoMaxGroups; ++i)
+    if (io.done[i]) cudaEventDestroy(io.done[i]);
+  if (io.begin) cudaEventDestroy(io.begin);
+  if (io.dev) cudaFree(io.dev);
+  if (io.pinned) cudaFreeHost(io.pinned);
+  delete[] io.order;
+  io = HostIo();
+}
+
 }  // namespace
 
 extern "C" {
+
+int fltop_enable_host_io(fltop_handle* h) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  if (h->cfg.max_chunk_frames > 0) return FLTOP_ERR_STATE;
+  if (h->io.ready) return FLTOP_OK;
+  DeviceGuard g;
+  cudaError_t e = g.enter(h->cfg.device);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  HostIo& io = h->io;
+  const size_t B = (size_t)h->cfg.max_batch, K = (size_t)h->cfg.beam_width;
+  const size_t L = (size_t)h->cfg.max_out_len;
+  const size_t n_logp = B * (size_t)h->cfg.max_frames * (size_t)h->cfg.vocab_size;
+  size_t off = 0;
+  const size_t o_logp = off; off += up(n_logp * 4);
+  const size_t o_len = off; off += up(B * 4);
+  const size_t o_tok = off; off += up(B * K * L * 4);
+  const size_t o_small = off; off += up(B * (2 * K + 2) * 4);
+  void* ptr = nullptr;
+  e = cudaMalloc(&ptr, off);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? FLTOP_ERR_OOM : cuda_fail(h, e);
+  }
+  io.dev = static_cast<unsigned char*>(ptr);
+  io.d_logp = reinterpret_cast<float*>(io.dev + o_logp);
+  io.d_lengths = reinterpret_cast<int32_t*>(io.dev + o_len);
+  io.d_tokens = reinterpret_cast<int32_t*>(io.dev + o_tok);
+  io.d_small = reinterpret_cast<int32_t*>(io.dev + o_small);
+  size_t poff = 0;
+  const size_t q_len = poff; poff += up(B * 4);
+  const size_t q_small = poff; poff += up(B * (2 * K + 2) * 4);
+  e = cudaHostAlloc(&ptr, poff, cudaHostAllocDefault);
+  if (e == cudaSuccess) {
+    io.pinned = static_cast<unsigned char*>(ptr);
+    io.p_lengths = reinterpret_cast<int32_t*>(io.pinned + q_len);
+    io.p_small = reinterpret_cast<int32_t*>(io.pinned + q_small);
+    io.order = new (std::nothrow) int32_t[B];
+    if (!io.order) e = cudaErrorMemoryAllocation;
+  }
+  for (int i = 0; i < kIoStreams && e == cudaSuccess; ++i) {
+    e = cudaStreamCreateWithFlags(&io.stream[i], cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&io.end[i], cudaEventDisableTiming);
+  }
+  for (int i = 0; i < kIoMaxGroups && e == cudaSuccess; ++i)
+    e = cudaEventCreateWithFlags(&io.done[i], cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&io.begin, cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    host_io_release(io);
+    return e == cudaErrorMemoryAllocation ? FLTOP_ERR_OOM : cuda_fail(h, e);
+  }
+  io.ready = true;
+  return FLTOP_OK;
+}
+
+int fltop_decode_host(fltop_handle* h, const float* h_logp, int64_t stride_b, int64_t stride_t,
+                      const int32_t* h_lengths, int32_t B, int32_t T, int32_t* h_tokens,
+                      int32_t* h_lens, float* h_scores, int32_t* h_nhyp, int32_t* h_status,
+                      void* cuda_stream) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  if (h->cfg.max_chunk_frames > 0 || !h->io.ready) return FLTOP_ERR_STATE;
+  if (B < 0 || T < 0) return FLTOP_ERR_INVALID_ARG;
+  if (B > h->cfg.max_batch || T > h->cfg.max_frames) return FLTOP_ERR_CAPACITY;
+  if (B > 0 && (!h_lengths || !h_tokens || !h_lens || !h_scores || !h_nhyp))
+    return FLTOP_ERR_INVALID_ARG;
+  if (B > 0 && T > 0 && (!h_logp || stride_t < h->cfg.vocab_size || stride_b < 0))
+    return FLTOP_ERR_INVALID_ARG;
+  HostIo& io = h->io;
+  io.h2d_bytes = io.d2h_bytes = 0;
+  if (B == 0) return FLTOP_OK;
+  DeviceGuard g;
+  cudaError_t e = g.enter(h->cfg.device);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t V = h->cfg.vocab_size, K = h->cfg.beam_width, L = h->cfg.max_out_len;
+
+  // The longest utterances go first: the call lasts as long as the longest frame chain, so that
+  // chain has to start as early as possible; everything else overlaps with it.
+  auto usable = [&](int32_t u) -> int64_t {
+    const int32_t len = h_lengths[u];
+    return (len < 0 || len > T) ? 0 : len;  // the kernel flags such an utterance itself
+  };
+  for (int32_t i = 0; i < B; ++i) io.order[i] = i;
+  std::stable_sort(io.order, io.order + B,
+                   [&](int32_t a, int32_t b) { return usable(a) > usable(b); });
+  for (int32_t i = 0; i < B; ++i) io.p_lengths[i] = h_lengths[io.order[i]];
+
+  // Groups of utterances, in slot order.  The first group (the longest utterances) is a
+  // quarter of the others: its copies are the head and the tail of the call that nothing
+  // overlaps with.
+  int32_t group = kIoGroupSize;
+  if ((B + group - 1) / group + 1 > kIoMaxGroups)
+    group = (B + kIoMaxGroups - 2) / (kIoMaxGroups - 1);
+  const int32_t first = std::min(B, std::max(1, group / 4));
+  const int32_t n_groups = 1 + (B - first + group - 1) / group;
+  auto group_begin = [&](int32_t gi) -> int32_t {
+    return gi == 0 ? 0 : std::min(B, first + (gi - 1) * group);
+  };
+
+  e = cudaEventRecord(io.begin, user);
+  for (int i = 0; i < n_groups && e == cudaSuccess; ++i)
+    e = cudaStreamWaitEvent(io.stream[i], io.begin, 0);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+
+  int rc = FLTOP_OK;
+  const int64_t row_pitch = (int64_t)T * V;  // device staging: [slot, T, V], this call's T
+  for (int32_t gi = 0; gi < n_groups && rc == FLTOP_OK; ++gi) {
+    const int32_t s0 = group_begin(gi), n = group_begin(gi + 1) - s0;
+    cudaStream_t st = io.stream[gi];
+    e = cudaMemcpyAsync(io.d_lengths + s0, io.p_lengths + s0, (size_t)n * 4,
+                        cudaMemcpyHostToDevice, st);
+    io.h2d_bytes += (int64_t)n * 4;
+    for (int32_t slot = s0; slot < s0 + n && e == cudaSuccess; ++slot) {
+      const int32_t u = io.order[slot];
+      const int64_t len = usable(u);
+      if (len == 0) continue;
+      float* dst = io.d_logp + (int64_t)slot * row_pitch;
+      const float* src = h_logp + (int64_t)u * stride_b;
+      if (stride_t == V) {
+        e = cudaMemcpyAsync(dst, src, (size_t)(len * V) * 4, cudaMemcpyHostToDevice, st);
+      } else {
+        e = cudaMemcpy2DAsync(dst, (size_t)V * 4, src, (size_t)stride_t * 4, (size_t)V * 4,
+                              (size_t)len, cudaMemcpyHostToDevice, st);
+      }
+      io.h2d_bytes += len * V * 4;
+    }
+    if (e != cudaSuccess) { rc = cuda_fail(h, e); break; }
+    int32_t* const small = io.d_small + (int64_t)s0 * (2 * K + 2);
+    rc = run_decode(h, io.d_logp + (int64_t)s0 * row_pitch, row_pitch, V, io.d_lengths + s0,
+                    nullptr, n, T, false, io.d_tokens + (int64_t)s0 * K * L, small,
+                    reinterpret_cast<float*>(small + (int64_t)n * K), small + (int64_t)2 * n * K,
+                    small + (int64_t)2 * n * K + n, st, s0, B);
+  }
+  // The small outputs come home in the order the groups will finish, shortest first: copies
+  // wait in the copy engine's queue in the order they were issued, and one that waits for a
+  // long kernel would hold up those behind it.
+  for (int32_t gi = n_groups - 1; gi >= 0 && rc == FLTOP_OK; --gi) {
+    const int32_t s0 = group_begin(gi), n = group_begin(gi + 1) - s0;
+    e = cudaMemcpyAsync(io.p_small + (int64_t)s0 * (2 * K + 2),
+                        io.d_small + (int64_t)s0 * (2 * K + 2), (size_t)(n * (2 * K + 2)) * 4,
+                        cudaMemcpyDeviceToHost, io.stream[gi]);
+    if (e == cudaSuccess) e = cudaEventRecord(io.done[gi], io.stream[gi]);
+    io.d2h_bytes += (int64_t)n * (2 * K + 2) * 4;
+    if (e != cudaSuccess) rc = cuda_fail(h, e);
+  }
+  h->last_B = B; h->last_T = T; h->last_stream = user; h->prof_valid = false;
+
+  // Results, shortest utterances (the last group) first: they are done long before the
+  // longest.  Only the tokens that exist cross the bus: hypotheses x longest hypothesis.
+  for (int32_t gi = n_groups - 1; gi >= 0 && rc == FLTOP_OK; --gi) {
+    const int32_t s0 = group_begin(gi), n = group_begin(gi + 1) - s0;
+    e = cudaEventSynchronize(io.done[gi]);
+    const int32_t* const small = io.p_small + (int64_t)s0 * (2 * K + 2);
+    const int32_t* const g_lens = small;
+    const float* const g_scores = reinterpret_cast<const float*>(small + (int64_t)n * K);
+    const int32_t* const g_nhyp = small + (int64_t)2 * n * K;
+    const int32_t* const g_status = g_nhyp + n;
+    for (int32_t slot = s0; slot < s0 + n && e == cudaSuccess; ++slot) {
+      const int32_t u = io.order[slot], i = slot - s0;
+      const int32_t nh = std::max(0, std::min<int32_t>(g_nhyp[i], (int32_t)K));
+      h_nhyp[u] = g_nhyp[i];
+      if (h_status) h_status[u] = g_status[i];
+      int32_t longest = 0;
+      for (int64_t k = 0; k < K; ++k) {
+        const int32_t len = g_lens[(int64_t)i * K + k];
+        h_lens[(int64_t)u * K + k] = len;
+        h_scores[(int64_t)u * K + k] = g_scores[(int64_t)i * K + k];
+        if (k < nh) longest = std::max(longest, len);
+      }
+      longest = (int32_t)std::min<int64_t>(longest, L);
+      if (nh > 0 && longest > 0) {
+        e = cudaMemcpy2DAsync(h_tokens + (int64_t)u * K * L, (size_t)L * 4,
+                              io.d_tokens + (int64_t)slot * K * L, (size_t)L * 4,
+                              (size_t)longest * 4, (size_t)nh, cudaMemcpyDeviceToHost,
+                              io.stream[gi]);
+        io.d2h_bytes += (int64_t)longest * nh * 4;
+      }
+    }
+    if (e != cudaSuccess) rc = cuda_fail(h, e);
+  }
+  // the caller's stream resumes after everything; the host returns with the outputs in place
+  for (int i = 0; i < n_groups; ++i) {
+    e = cudaEventRecord(io.end[i], io.stream[i]);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(user, io.end[i], 0);
+    if (e != cudaSuccess && rc == FLTOP_OK) rc = cuda_fail(h, e);
+  }
+  e = cudaStreamSynchronize(user);
+  if (e != cudaSuccess && rc == FLTOP_OK) rc = cuda_fail(h, e);
+  if (rc != FLTOP_OK)  // leave nothing of this call in flight
+    for (int i = 0; i < n_groups; ++i) cudaStreamSynchronize(io.stream[i]);
+  return rc;
+}
+
+int fltop_last_host_io_bytes(const fltop_handle* h, int64_t* out) {
+  if (!h || !out) return FLTOP_ERR_INVALID_ARG;
+  out[0] = h->io.h2d_bytes;
+  out[1] = h->io.d2h_bytes;
+  return FLTOP_OK;
+}
 
 size_t fltop_workspace_size(const fltop_config* cfg) {
   if (!config_ok(cfg)) return 0;
@@ -298,6 +545,7 @@ int fltop_destroy(fltop_handle* h) {
   if (g.enter(h->cfg.device) != cudaSuccess) rc = FLTOP_ERR_CUDA;
   for (int i = 0; i < 3; ++i)
     if (h->ev[i]) cudaEventDestroy(h->ev[i]);
+  host_io_release(h->io);
   if (h->owns_workspace && h->ws && cudaFree(h->ws) != cudaSuccess) rc = FLTOP_ERR_CUDA;
   cudaGetLastError();
   delete h;

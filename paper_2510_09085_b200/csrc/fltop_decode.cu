@@ -1350,10 +1350,11 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int blocks = p.co_resident > p.B ? p.co_resident : p.B;
   int nt = p.block_threads > 0
                ? p.block_threads
-               : decode_block_threads(p.K, p.V, p.pruning != 0, p.top_n, p.B <= sms);
-  if (p.block_threads <= 0 && nt > 512 && p.pruning && p.B > sms) {
+               : decode_block_threads(p.K, p.V, p.pruning != 0, p.top_n, blocks <= sms);
+  if (p.block_threads <= 0 && nt > 512 && p.pruning && blocks > sms) {
     // more utterances than SMs: two blocks of 512 threads per SM overlap their frame chains
     // better than one block of 1024 (measured on the subword shape, B = 256)
     nt = 512;
@@ -1363,10 +1364,10 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   if (nt > kMaxThreads) nt = kMaxThreads;
   const size_t bytes = decode_smem_bytes(p.K, p.V);
   switch (pick_variant(p.K, p.V)) {
-    case kCharBeam64: launch_variant<64, 32>(p, nt, bytes, p.B <= sms, s); break;
-    case kSubwordBeam64: launch_variant<64, 1024>(p, nt, bytes, p.B <= sms, s); break;
-    case kWideBeam: launch_variant<-1, 0>(p, nt, bytes, p.B <= sms, s); break;
-    default: launch_variant<0, 0>(p, nt, bytes, p.B <= sms, s); break;
+    case kCharBeam64: launch_variant<64, 32>(p, nt, bytes, blocks <= sms, s); break;
+    case kSubwordBeam64: launch_variant<64, 1024>(p, nt, bytes, blocks <= sms, s); break;
+    case kWideBeam: launch_variant<-1, 0>(p, nt, bytes, blocks <= sms, s); break;
+    default: launch_variant<0, 0>(p, nt, bytes, blocks <= sms, s); break;
   }
   return cudaGetLastError();
 }

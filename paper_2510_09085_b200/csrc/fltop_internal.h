@@ -51,6 +51,9 @@ struct DecodeParams {
   int32_t streaming;        // 0: reset at entry, no state kept.  1: state loaded / stored
   int32_t emit_default;     // streaming with flags == null: emit results?
   int32_t block_threads;    // 0 = choose from K, V and whether pruning is on
+  int32_t co_resident;      // utterance blocks on the GPU at the same time as this launch's,
+                            // its own included (0 = just its own B): launches of one batch
+                            // split over several streams size their blocks for the whole batch
   int32_t pruning;          // 1 when R is large enough that few tokens survive a frame
   int32_t top_n;            // survivors per frame are capped at this (0: no cap)
   float beam_threshold;     // kept prefixes score at least best - beam_threshold (<= 0: off)

@@ -71,6 +71,10 @@ def test_null_arguments(bd):
     assert bd.lib().fltop_prune(None, None, 0, 0, None, 0, 0, None, None, None) == \
         bd.FLTOP_ERR_INVALID_ARG
     assert bd.lib().fltop_set_profiling(None, 1) == bd.FLTOP_ERR_INVALID_ARG
+    assert bd.lib().fltop_enable_host_io(None) == bd.FLTOP_ERR_INVALID_ARG
+    assert bd.lib().fltop_decode_host(None, None, 0, 0, None, 0, 0, None, None, None, None, None,
+                                      None) == bd.FLTOP_ERR_INVALID_ARG
+    assert bd.lib().fltop_last_host_io_bytes(None, None) == bd.FLTOP_ERR_INVALID_ARG
     assert bd.lib().fltop_launch_count(None) == 0
 
 
