@@ -23,6 +23,11 @@ import time
 
 import numpy as np
 
+# fltop_decode_host runs a batch as up to 16 groups on as many streams; with CUDA's default of 8
+# hardware connections streams share queues and wait on one another's work.  Read by the
+# driver when the process creates its CUDA context.
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
+
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)

@@ -129,7 +129,9 @@ int fltop_enable_host_io(fltop_handle* h);
  * h_lens, h_scores, h_nhyp and (if not NULL) h_status are written in full.
  * The work is ordered after what `cuda_stream` held at the call and `cuda_stream` waits for
  * it; unlike the device-pointer calls this one RETURNS ONLY WHEN THE OUTPUTS ARE IN HOST
- * MEMORY.  Results are those of fltop_decode, bit for bit.  FLTOP_ERR_STATE unless
+ * MEMORY.  Results are those of fltop_decode, bit for bit.  (Up to 16 of the handle's streams
+ * are busy at once; a process that leaves CUDA_DEVICE_MAX_CONNECTIONS at its default of 8 lets
+ * them share hardware queues, which costs a few per cent.)  FLTOP_ERR_STATE unless
  * fltop_enable_host_io succeeded on this handle. */
 int fltop_decode_host(fltop_handle* h, const float* h_logp, int64_t stride_b, int64_t stride_t,
                       const int32_t* h_lengths, int32_t B, int32_t T, int32_t* h_tokens,
