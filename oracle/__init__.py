@@ -65,7 +65,9 @@ def _load():
         lib.oracle_decode_opt.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_void_p, c.c_int,
                                           c.c_int, c.c_int, c.c_int, c.c_int, c.c_float, c.c_int,
                                           c.c_double, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p,
-                                          c.c_void_p, c.c_void_p, c.c_void_p]
+                                          c.c_void_p, c.c_void_p, c.c_void_p, c.c_int]
+        lib.oracle_stream_merge_max.restype = None
+        lib.oracle_stream_merge_max.argtypes = [c.c_void_p, c.c_int]
         lib.oracle_decode.restype = None
         lib.oracle_decode.argtypes = [c.c_void_p, c.c_int64, c.c_int64, c.c_void_p, c.c_int,
                                       c.c_int, c.c_int, c.c_int, c.c_int, c.c_float, c.c_int,
@@ -111,10 +113,13 @@ class DecodeResult:
 
 
 def decode(lp: np.ndarray, lengths, blank: int, K: int, r: float, max_len: int | None = None,
-           want_masks: bool = False, top_n: int = 0, beam_threshold: float = 0.0) -> DecodeResult:
+           want_masks: bool = False, top_n: int = 0, beam_threshold: float = 0.0,
+           merge_max: bool = False) -> DecodeResult:
     """Frame-pruned CTC prefix beam search of a padded batch ``lp`` [B,T,V].
 
-    ``top_n`` and ``beam_threshold`` are N and beam_threshold of Algorithm 1 (0 = off)."""
+    ``top_n`` and ``beam_threshold`` are N and beam_threshold of Algorithm 1 (0 = off).
+    ``merge_max``: masses are combined by max instead of log-sum (Algorithm 1's literal
+    score' = score + logit: a prefix scores as its best single alignment)."""
     lp = np.ascontiguousarray(lp, dtype=np.float32)
     B, T, V = lp.shape
     lengths = np.ascontiguousarray(lengths, dtype=np.int32)
@@ -128,7 +133,7 @@ def decode(lp: np.ndarray, lengths, blank: int, K: int, r: float, max_len: int |
     _load().oracle_decode_opt(_ptr(lp), T * V, V, _ptr(lengths), B, T, V, blank, K,
                               float(np.float32(r)), int(top_n), float(beam_threshold), L,
                               _ptr(tokens), _ptr(lens), _ptr(scores), _ptr(nhyp), _ptr(keep),
-                              _ptr(counts))
+                              _ptr(counts), int(bool(merge_max)))
     return DecodeResult(tokens, lens, scores, nhyp,
                         None if keep is None else keep.astype(bool), counts)
 
@@ -137,10 +142,11 @@ class Stream:
     """One utterance decoded incrementally; state persists between ``feed`` calls."""
 
     def __init__(self, V: int, blank: int, K: int, r: float, top_n: int = 0,
-                 beam_threshold: float = 0.0):
+                 beam_threshold: float = 0.0, merge_max: bool = False):
         self.V, self.K = V, K
         self._h = _load().oracle_stream_create(V, blank, K, float(np.float32(r)))
         _load().oracle_stream_options(self._h, int(top_n), float(beam_threshold))
+        _load().oracle_stream_merge_max(self._h, int(bool(merge_max)))
 
     def feed(self, lp: np.ndarray):
         lp = np.ascontiguousarray(lp, dtype=np.float32).reshape(-1, self.V)

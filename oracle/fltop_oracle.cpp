@@ -28,6 +28,12 @@
 //   * beam_threshold (second argument of SelectTopK): after the best beam_size
 //     candidates are chosen, those scoring below best - beam_threshold are
 //     dropped.  beam_threshold <= 0 means no such cut.
+// A third option restates Algorithm 1's score update literally: it writes
+// score' = score + logit for a candidate and never sums over the alignments
+// of a prefix, which is what decoders of the flashlight family do when their
+// log-add option is off.  With merge_max every combination of two masses
+// below (equal prefixes in B'.add, blank and non-blank mass of a prefix) takes
+// the larger one, so a prefix's score is that of its single best alignment.
 //
 // A prefix is identified by its full token sequence.  Sequences are stored in
 // a trie whose child table is never pruned, so one node id corresponds to
@@ -58,7 +64,6 @@ double log_add(double a, double b) {
 struct Mass {
   double pb = NEG_INF;   // log-mass of alignments of this prefix ending in blank
   double pnb = NEG_INF;  // ... ending in the prefix's last token
-  double total() const { return log_add(pb, pnb); }
 };
 
 struct TrieNode {
@@ -71,6 +76,7 @@ struct Decoder {
   int V, blank, K;
   int top_n = 0;                 // 0: no cap
   double beam_threshold = 0.0;   // <= 0: no cut
+  bool merge_max = false;        // combine masses by max instead of log-sum
   float log_r;
   std::vector<TrieNode> nodes;                  // node 0 = empty prefix
   std::map<std::pair<int, int>, int> child;     // (parent node, token) -> node
@@ -91,6 +97,9 @@ struct Decoder {
     beam.assign(1, std::make_pair(0, m));
     frames_seen = 0;
   }
+
+  double combine(double a, double b) const { return merge_max ? std::max(a, b) : log_add(a, b); }
+  double total(const Mass& m) const { return combine(m.pb, m.pnb); }
 
   int child_of(int p, int c) {
     auto key = std::make_pair(p, c);
@@ -143,22 +152,22 @@ struct Decoder {
     for (const auto& entry : beam) {
       int node = entry.first;
       const Mass& m = entry.second;
-      double tot = m.total();
+      double tot = total(m);
       int last = nodes[node].token;  // -1 for the empty prefix
       if (keep[blank]) {
         Mass& s = next[node];
-        s.pb = log_add(s.pb, tot + (double)lp[blank]);
+        s.pb = combine(s.pb, tot + (double)lp[blank]);
       }
       if (last >= 0 && keep[last]) {
         Mass& s = next[node];
-        s.pnb = log_add(s.pnb, m.pnb + (double)lp[last]);
+        s.pnb = combine(s.pnb, m.pnb + (double)lp[last]);
       }
       for (int c = 0; c < V; ++c) {
         if (c == blank || !keep[c]) continue;
         // a repeated token starts a new symbol only after a blank
         double from = (c == last) ? m.pb : tot;
         Mass& s = next[child_of(node, c)];
-        s.pnb = log_add(s.pnb, from + (double)lp[c]);
+        s.pnb = combine(s.pnb, from + (double)lp[c]);
       }
     }
 
@@ -169,7 +178,7 @@ struct Decoder {
     };
     std::vector<Cand> cands;
     for (const auto& kv : next) {
-      double t = kv.second.total();
+      double t = total(kv.second);
       if (t == NEG_INF) continue;
       cands.push_back(Cand{kv.first, kv.second, t});
     }
@@ -212,6 +221,7 @@ void oracle_stream_options(void* h, int top_n, double beam_threshold) {
   ((Decoder*)h)->top_n = top_n;
   ((Decoder*)h)->beam_threshold = beam_threshold;
 }
+void oracle_stream_merge_max(void* h, int merge_max) { ((Decoder*)h)->merge_max = merge_max != 0; }
 // Survivor mask with the top-N cap.
 void oracle_prune_topn(const float* lp, int64_t n_frames, int V, float r, int top_n, uint8_t* keep,
                        int32_t* counts) {
@@ -248,7 +258,7 @@ int oracle_stream_results(void* h, int32_t* tokens, int32_t* lens, double* score
     if (lens) lens[k] = (int)s.size();
     if (tokens)
       for (int i = 0; i < (int)s.size() && i < max_len; ++i) tokens[(int64_t)k * max_len + i] = s[i];
-    if (scores) scores[k] = d->beam[k].second.total();
+    if (scores) scores[k] = d->total(d->beam[k].second);
     if (pb) pb[k] = d->beam[k].second.pb;
     if (pnb) pnb[k] = d->beam[k].second.pnb;
   }
@@ -262,11 +272,13 @@ int oracle_stream_results(void* h, int32_t* tokens, int32_t* lens, double* score
 void oracle_decode_opt(const float* lp, int64_t stride_b, int64_t stride_t, const int32_t* lengths,
                        int B, int T, int V, int blank, int K, float r, int top_n,
                        double beam_threshold, int max_len, int32_t* tokens, int32_t* lens,
-                       double* scores, int32_t* nhyp, uint8_t* keep, int32_t* counts) {
+                       double* scores, int32_t* nhyp, uint8_t* keep, int32_t* counts,
+                       int merge_max) {
   for (int b = 0; b < B; ++b) {
     Decoder d(V, blank, K, r);
     d.top_n = top_n;
     d.beam_threshold = beam_threshold;
+    d.merge_max = merge_max != 0;
     int len = lengths[b];
     if (len < 0 || len > T) {
       nhyp[b] = 0;
@@ -289,7 +301,7 @@ void oracle_decode(const float* lp, int64_t stride_b, int64_t stride_t, const in
                    int B, int T, int V, int blank, int K, float r, int max_len, int32_t* tokens,
                    int32_t* lens, double* scores, int32_t* nhyp, uint8_t* keep, int32_t* counts) {
   oracle_decode_opt(lp, stride_b, stride_t, lengths, B, T, V, blank, K, r, 0, 0.0, max_len, tokens,
-                    lens, scores, nhyp, keep, counts);
+                    lens, scores, nhyp, keep, counts, 0);
 }
 
 }  // extern "C"

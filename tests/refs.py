@@ -23,11 +23,13 @@ def collapse(path, blank):
     return tuple(out)
 
 
-def brute_force(lp: np.ndarray, blank: int, keep: np.ndarray | None = None) -> dict:
+def brute_force(lp: np.ndarray, blank: int, keep: np.ndarray | None = None,
+                best_alignment: bool = False) -> dict:
     """log P(labelling) for every labelling, by enumerating all V**T alignments.
 
     ``keep`` [T,V] (bool) restricts each frame to its surviving tokens.
-    Probabilities are summed in float64 with math.fsum.
+    Probabilities are summed in float64 with math.fsum.  ``best_alignment``: the
+    log-probability of the labelling's single most probable alignment instead of their sum.
     """
     T, V = lp.shape
     terms: dict = {}
@@ -39,7 +41,8 @@ def brute_force(lp: np.ndarray, blank: int, keep: np.ndarray | None = None) -> d
         for t, c in enumerate(path):
             w *= p[t, c]
         terms.setdefault(collapse(path, blank), []).append(w)
-    return {k: (math.log(s) if (s := math.fsum(v)) > 0 else -math.inf) for k, v in terms.items()}
+    total = max if best_alignment else math.fsum
+    return {k: (math.log(s) if (s := total(v)) > 0 else -math.inf) for k, v in terms.items()}
 
 
 def greedy(lp: np.ndarray, blank: int):
@@ -58,8 +61,9 @@ def _lse(a, b):
 class PyPrefixSearch:
     """Dictionary-keyed CTC prefix beam search, optional per-frame survivor sets."""
 
-    def __init__(self, blank: int, K: int, beam_threshold: float = 0.0):
+    def __init__(self, blank: int, K: int, beam_threshold: float = 0.0, merge_max: bool = False):
         self.blank, self.K, self.beam_threshold = blank, K, beam_threshold
+        self._mix = max if merge_max else _lse
         self.beam = {(): (0.0, -math.inf)}
         self.revivals = 0          # prefixes that re-entered the beam after leaving it
         self._ever = {()}
@@ -70,10 +74,10 @@ class PyPrefixSearch:
 
         def add(key, which, val):
             pb, pnb = nxt.get(key, (-math.inf, -math.inf))
-            nxt[key] = (_lse(pb, val), pnb) if which == 0 else (pb, _lse(pnb, val))
+            nxt[key] = (self._mix(pb, val), pnb) if which == 0 else (pb, self._mix(pnb, val))
 
         for seq, (pb, pnb) in self.beam.items():
-            tot = _lse(pb, pnb)
+            tot = self._mix(pb, pnb)
             for c in survivors:
                 v = float(lp_row[c])
                 if c == self.blank:
@@ -83,12 +87,13 @@ class PyPrefixSearch:
                     add(seq + (c,), 1, pb + v)
                 else:
                     add(seq + (c,), 1, tot + v)
-        items = [(k, v) for k, v in nxt.items() if _lse(*v) > -math.inf]
-        items.sort(key=lambda kv: (-_lse(*kv[1]), len(kv[0]), kv[0]))
+        mix = self._mix
+        items = [(k, v) for k, v in nxt.items() if mix(*v) > -math.inf]
+        items.sort(key=lambda kv: (-mix(*kv[1]), len(kv[0]), kv[0]))
         items = items[: self.K]
         if self.beam_threshold > 0 and items:
-            floor = _lse(*items[0][1]) - self.beam_threshold
-            items = [kv for kv in items if _lse(*kv[1]) >= floor]
+            floor = mix(*items[0][1]) - self.beam_threshold
+            items = [kv for kv in items if mix(*kv[1]) >= floor]
         self.beam = dict(items)
         now = set(self.beam)
         self.revivals += len([s for s in now if s in self._ever and s not in self._prev])
@@ -96,7 +101,7 @@ class PyPrefixSearch:
         self._prev = now
 
     def results(self):
-        out = [(k, _lse(*v)) for k, v in self.beam.items()]
+        out = [(k, self._mix(*v)) for k, v in self.beam.items()]
         out.sort(key=lambda kv: (-kv[1], len(kv[0]), kv[0]))
         return out
 
@@ -107,13 +112,13 @@ def top_n_tokens(row: np.ndarray, n: int):
 
 
 def py_decode(lp: np.ndarray, blank: int, K: int, log_r: np.float32 | None, top_n: int = 0,
-              beam_threshold: float = 0.0):
+              beam_threshold: float = 0.0, merge_max: bool = False):
     """Decode one utterance [T,V]; ``log_r`` None means no survivor test at all.
 
     ``top_n`` > 0: only the top_n most probable tokens of a frame are candidates for the
     survivor test.  ``beam_threshold`` > 0: kept prefixes score at least best - beam_threshold."""
     T, V = lp.shape
-    s = PyPrefixSearch(blank, K, beam_threshold)
+    s = PyPrefixSearch(blank, K, beam_threshold, merge_max)
     for t in range(T):
         cand = top_n_tokens(lp[t], top_n) if top_n > 0 else range(V)
         if log_r is None:

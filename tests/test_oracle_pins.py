@@ -316,3 +316,53 @@ def test_streaming_with_options_equals_one_shot():
     for a, b in [(0, 7), (7, 8), (8, 33), (33, 50)]:
         st.feed(lp[a:b])
     assert st.results() == full
+
+
+# ---------------------------------------------------------------- merge by max (best alignment)
+@pytest.mark.parametrize("seed,T,V,blank,r", [(40, 4, 3, 0, 0.0), (41, 6, 3, 1, 0.0),
+                                              (42, 6, 4, 2, 0.0), (43, 6, 4, 0, 0.3),
+                                              (44, 5, 4, 3, 0.6)])
+def test_merge_max_scores_equal_the_best_alignment_of_each_labelling(seed, T, V, blank, r):
+    lp = _rand_logp(seed, T, V, sharp=1.0)
+    res = oracle.decode(lp[None], [T], blank, 10000, r, want_masks=True, merge_max=True)
+    got = dict(res.hyps(0))
+    exact = {k: v for k, v in brute_force(lp, blank, res.keep[0], best_alignment=True).items()
+             if v > -math.inf}
+    assert set(got) == set(exact)
+    for seq, v in exact.items():
+        assert got[seq] == pytest.approx(v, abs=1e-9)
+    # the sum over alignments can only be larger, and is for a labelling with several of them
+    summed = dict(oracle.decode(lp[None], [T], blank, 10000, r).hyps(0))
+    assert all(summed[s] >= got[s] - 1e-12 for s in got)
+    assert any(summed[s] > got[s] + 1e-6 for s in got)
+
+
+@pytest.mark.parametrize("K", [1, 3, 50])
+def test_merge_max_best_hypothesis_is_the_best_path_whatever_the_beam(K):
+    # under max the best partial alignment is the best-scoring prefix at every frame, so it is
+    # never cut: top-1 = collapse of the frame-wise argmax, score = sum of the row maxima
+    lp = _rand_logp(45, 60, 7, sharp=2.0)
+    top = oracle.decode(lp[None], [60], 0, K, 0.0, merge_max=True).hyps(0)[0]
+    assert top[0] == greedy(lp, 0)
+    assert top[1] == pytest.approx(float(lp.astype(np.float64).max(axis=1).sum()), abs=1e-9)
+
+
+@pytest.mark.parametrize("K,r,n,theta", [(4, 0.05, 0, 0.0), (8, 0.0, 0, 0.0), (6, 0.01, 3, 4.0)])
+def test_merge_max_matches_the_second_implementation(K, r, n, theta):
+    em, ln = W.make_small(46, 3, 30, 50, 6)
+    res = oracle.decode(em, ln, 0, K, r, top_n=n, beam_threshold=theta, merge_max=True)
+    for b in range(3):
+        ref = py_decode(em[b, : ln[b]], 0, K, oracle.log_r(r), top_n=n, beam_threshold=theta,
+                        merge_max=True)
+        got, want = res.hyps(b), ref.results()
+        assert [s for s, _ in got] == [s for s, _ in want]
+        np.testing.assert_allclose([v for _, v in got], [v for _, v in want], atol=1e-9)
+
+
+def test_merge_max_streaming_equals_one_shot():
+    lp = _rand_logp(47, 40, 8, sharp=1.0)
+    full = oracle.decode(lp[None], [40], 0, 5, 0.02, merge_max=True).hyps(0)
+    st = oracle.Stream(8, 0, 5, 0.02, merge_max=True)
+    for a, b in [(0, 1), (1, 19), (19, 40)]:
+        st.feed(lp[a:b])
+    assert st.results() == full
