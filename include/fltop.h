@@ -80,6 +80,10 @@ typedef struct {
                              best prefixes of a frame, those scoring below best -
                              beam_threshold are dropped, so a beam can hold fewer than
                              beam_width prefixes.  <= 0 = no such cut */
+  int32_t merge_max;      /* 0: candidates naming the same prefix, and a prefix' blank and
+                             non-blank mass, are combined by log-sum (a prefix scores as the
+                             sum over its alignments).  1: by max, Algorithm 1's literal
+                             score' = score + logit: a prefix scores as its best alignment */
   int32_t device;         /* CUDA device ordinal */
   void* workspace;        /* optional DEVICE memory, 256-byte aligned, for all of the
                              handle's scratch; NULL = the library allocates it */

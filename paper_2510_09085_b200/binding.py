@@ -32,7 +32,8 @@ class fltop_config(C.Structure):
     _fields_ = [("vocab_size", C.c_int32), ("blank_id", C.c_int32), ("beam_width", C.c_int32),
                 ("threshold_r", C.c_float), ("max_batch", C.c_int32), ("max_frames", C.c_int32),
                 ("max_chunk_frames", C.c_int32), ("max_out_len", C.c_int32),
-                ("top_n", C.c_int32), ("beam_threshold", C.c_float), ("device", C.c_int32),
+                ("top_n", C.c_int32), ("beam_threshold", C.c_float), ("merge_max", C.c_int32),
+                ("device", C.c_int32),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
@@ -104,10 +105,11 @@ def status_string(code: int) -> str:
 
 def make_config(vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                 max_chunk_frames=0, max_out_len=None, device=0, workspace=0, workspace_bytes=0,
-                top_n=0, beam_threshold=0.0) -> fltop_config:
+                top_n=0, beam_threshold=0.0, merge_max=0) -> fltop_config:
     return fltop_config(vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                         max_chunk_frames, max_frames if max_out_len is None else max_out_len,
-                        top_n, beam_threshold, device, workspace or None, workspace_bytes)
+                        top_n, beam_threshold, int(merge_max), device, workspace or None,
+                        workspace_bytes)
 
 
 def fltop_workspace_size(cfg: fltop_config) -> int:
@@ -171,10 +173,11 @@ class Decoder:
     """Owns one handle plus the output tensors; thin convenience over the C calls."""
 
     def __init__(self, vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
-                 max_chunk_frames=0, max_out_len=None, device=0, top_n=0, beam_threshold=0.0):
+                 max_chunk_frames=0, max_out_len=None, device=0, top_n=0, beam_threshold=0.0,
+                 merge_max=False):
         self.cfg = make_config(vocab_size, blank_id, beam_width, threshold_r, max_batch,
                                max_frames, max_chunk_frames, max_out_len, device, top_n=top_n,
-                               beam_threshold=beam_threshold)
+                               beam_threshold=beam_threshold, merge_max=int(bool(merge_max)))
         code, self.h = fltop_create(self.cfg)
         if code != FLTOP_OK:
             self.h = None

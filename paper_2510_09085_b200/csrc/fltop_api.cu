@@ -81,6 +81,7 @@ bool config_ok(const fltop_config* c) {
   if (c->max_chunk_frames < 0 || c->max_chunk_frames > c->max_frames) return false;
   if (c->top_n < 0) return false;
   if (c->beam_threshold != c->beam_threshold) return false;  // NaN
+  if (c->merge_max != 0 && c->merge_max != 1) return false;
   if (c->device < 0) return false;
   if ((int64_t)(c->beam_width + 1) * c->max_frames + 2 > (int64_t)std::numeric_limits<int32_t>::max())
     return false;
@@ -160,6 +161,7 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
   dp.block_threads = h->block_threads; dp.co_resident = co_resident; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
   dp.top_n = h->cfg.top_n; dp.beam_threshold = h->cfg.beam_threshold;
+  dp.merge_max = h->cfg.merge_max;
   dp.counts = pp.counts; dp.entries = pp.entries;
   dp.nodes = h->nodes + (int64_t)slot0 * h->nodes_per_utt;
   const bool fuse = h->fusion != 0 && T > 0 && decode_can_prune(h->cfg.vocab_size);

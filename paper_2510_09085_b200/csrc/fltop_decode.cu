@@ -393,7 +393,8 @@ __device__ __forceinline__ void divmod_small(int e, int d, float inv_d, int& q, 
 // constant; 0: laid out for the K and V of the call; -1: likewise, for wide beams (a crowded
 // cut bin is split a second time, and the warps are shared out between the two kinds of
 // candidate anew every frame).
-// BT: beam_threshold is on (the exact best score of every frame is tracked).
+// BT: an option of Algorithm 1 beyond N and R is on - beam_threshold (the exact best score of
+// every frame is tracked) and / or merging by max instead of log-sum.
 template <int MAXT, int KMAX, int VMAX, bool BT>
 __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
@@ -444,7 +445,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   bool is_ext = !is_chore && !is_stay;
   int xl = tid - NS;                         // index among the ext lanes
   const bool warp_scans = NT <= kSmallBlock;
-  constexpr bool use_bt = BT;
+  // the options live in instantiations of their own (BT): the default one has neither
+  const bool use_bt = BT && p.beam_threshold > 0.f;
+  const bool use_max = BT && p.merge_max != 0;
 
   int len = p.lengths[b];
   unsigned flags = 3u;
@@ -710,7 +713,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           const Hot pe = hc[pq];
           const float dup = ((pe.last == e.last) ? pe.pb : pe.tot) + le;
           if (dup != neg_inf()) {  // the parent's extension by last(q) names this prefix
-            npnb = lse2(npnb, dup);
+            npnb = use_max ? fmaxf(npnb, dup) : lse2(npnb, dup);
             atomicSub(&hist[score_bin(dup)], 1u);
             const int jp = jpos[e.last];  // position among all survivors -> among non-blank
             const int ed = pq * Snb + jp - ((blank_j >= 0 && jp > blank_j) ? 1 : 0);
@@ -720,7 +723,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       }
       st_pb[q] = npb;
       st_pnb[q] = npnb;
-      const float tot = lse2(npb, npnb);
+      // a prefix' blank and non-blank mass: summed, or (merge_max) the better one
+      const float tot = use_max ? fmaxf(npb, npnb) : lse2(npb, npnb);
       st_tot[q] = tot;
       if (tot != neg_inf()) count(tot);
       return tot;
@@ -1317,7 +1321,7 @@ cudaError_t prepare_variant(int bytes) {
 }
 template <int KMAX, int VMAX>
 void launch_variant(const DecodeParams& p, int nt, size_t bytes, bool alone, cudaStream_t s) {
-  const bool bt = p.beam_threshold > 0.f;
+  const bool bt = p.beam_threshold > 0.f || p.merge_max != 0;  // an option is on
   if (nt <= kSmallBlock) {
     if (bt) decode_kernel<kSmallBlock, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
     else decode_kernel<kSmallBlock, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);

@@ -57,6 +57,7 @@ struct DecodeParams {
   int32_t pruning;          // 1 when R is large enough that few tokens survive a frame
   int32_t top_n;            // survivors per frame are capped at this (0: no cap)
   float beam_threshold;     // kept prefixes score at least best - beam_threshold (<= 0: off)
+  int32_t merge_max;        // 1: masses are combined by max instead of log-sum
   int32_t* counts;          // [B*T] survivors per frame (a kernel that prunes itself leaves
                             // each utterance's total in its first frame's place, zeros after)
   const Survivor* entries;  // [B*T*V]

@@ -31,16 +31,17 @@ def test_top_n_survivors_bit_exact(V, r, n):
     d.close()
 
 
-def _compare(em, ln, K, r, top_n=0, theta=0.0, frac=0.0):
+def _compare(em, ln, K, r, top_n=0, theta=0.0, frac=0.0, merge_max=False):
     """Every utterance against the oracle.  With a beam threshold the two sides may differ on
     hypotheses within the tolerance of the threshold, so the beams are compared there as sets."""
     B, T, V = em.shape
-    d = _binding().Decoder(V, 0, K, r, B, T, top_n=top_n, beam_threshold=theta)
+    d = _binding().Decoder(V, 0, K, r, B, T, top_n=top_n, beam_threshold=theta,
+                           merge_max=merge_max)
     d.decode(_dev(em), _dev(ln))
     torch.cuda.synchronize()
     assert (d.status.cpu().numpy()[:B] == 0).all()
     st = d.last_call_stats()
-    res = oracle.decode(em, ln, 0, K, r, top_n=top_n, beam_threshold=theta)
+    res = oracle.decode(em, ln, 0, K, r, top_n=top_n, beam_threshold=theta, merge_max=merge_max)
     res.mean_live = st["live_hypotheses_sum"] / max(1, st["frames"])
     for b in range(B):
         g, o = d.hyps(b), res.hyps(b)
@@ -122,3 +123,55 @@ def test_streaming_with_options_equals_one_shot():
     assert torch.equal(one.nhyp[:B], st.nhyp[:B]) and torch.equal(one.scores[:B], st.scores[:B])
     for b in range(B):
         assert one.hyps(b) == st.hyps(b)
+
+
+# ------------------------------------------------------------------ merge by max
+@pytest.mark.parametrize("V,K,r,n,theta", [(32, 50, 1e-3, 0, 0.0), (32, 20, 0.0, 0, 0.0),
+                                           (32, 8, 0.01, 4, 0.0), (1024, 16, 1e-3, 0, 0.0),
+                                           (32, 300, 1e-3, 0, 0.0), (12, 10, 0.02, 3, 6.0)])
+def test_decode_with_merge_max_matches_oracle(V, K, r, n, theta):
+    em, ln = W.make_small(1500 + V + K, 5, 30, 110, V)
+    _compare(em, ln, K, r, top_n=n, theta=theta, merge_max=True)
+
+
+def test_merge_max_best_hypothesis_is_the_best_path():
+    # closed form: under max the best prefix is the collapse of the frame-wise argmax and its
+    # score the sum of the row maxima, at any beam width
+    em, ln = W.make_small(1600, 6, 40, 160, 32)
+    for K in (1, 7, 50):
+        d = _binding().Decoder(32, 0, K, 0.0, 6, em.shape[1], merge_max=True)
+        d.decode(_dev(em), _dev(ln))
+        torch.cuda.synchronize()
+        for b in range(6):
+            row = em[b, : ln[b]]
+            seq, sc = d.hyps(b)[0]
+            path, prev = [], None
+            for c in row.argmax(axis=1):
+                if c != prev and c != 0:
+                    path.append(int(c))
+                prev = c
+            assert list(seq) == path
+            assert abs(sc - float(row.astype(np.float64).max(axis=1).sum())) <= TOL
+        d.close()
+
+
+def test_merge_max_streaming_equals_one_shot():
+    em, ln = W.make_small(1700, 4, 20, 90, 32)
+    T = em.shape[1]
+    one = _binding().Decoder(32, 0, 12, 1e-2, 4, T, merge_max=True)
+    one.decode(_dev(em), _dev(ln))
+    st = _binding().Decoder(32, 0, 12, 1e-2, 4, T, max_chunk_frames=8, merge_max=True)
+    x = _dev(em)
+    n_chunks = (T + 7) // 8
+    for i in range(n_chunks):
+        chunk = torch.zeros((4, 8, 32), dtype=torch.float32, device="cuda")
+        w = min(8, T - 8 * i)
+        chunk[:, :w] = x[:, 8 * i: 8 * i + w]
+        clen = np.clip(ln - 8 * i, 0, 8).astype(np.int32)
+        flags = np.full(4, (1 if i == 0 else 0) | (2 if i == n_chunks - 1 else 0), dtype=np.uint8)
+        st.stream_step(chunk, _dev(clen), _dev(flags))
+    torch.cuda.synchronize()
+    for b in range(4):
+        assert one.hyps(b) == st.hyps(b)
+    one.close()
+    st.close()
