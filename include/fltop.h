@@ -49,6 +49,16 @@ enum {
                                 handle or the reverse) */
 };
 
+/* How the emissions are stored (fltop_config.emission_dtype).  Half-precision values are
+ * widened to float32 (exactly) as they are loaded; everything else, the pruning comparison
+ * included, is the float32 arithmetic described below.  Every `logp` / `chunk` pointer of
+ * this header points to elements of the handle's emission_dtype; strides count elements. */
+enum {
+  FLTOP_EMISSION_F32 = 0,
+  FLTOP_EMISSION_F16 = 1,    /* IEEE binary16 */
+  FLTOP_EMISSION_BF16 = 2    /* bfloat16 */
+};
+
 /* Per-utterance device status bits written to d_status (0 = fine). */
 enum {
   FLTOP_ST_BAD_LENGTH = 1,   /* length < 0 or > T: utterance skipped, nhyp = 0 */
@@ -84,6 +94,7 @@ typedef struct {
                              non-blank mass, are combined by log-sum (a prefix scores as the
                              sum over its alignments).  1: by max, Algorithm 1's literal
                              score' = score + logit: a prefix scores as its best alignment */
+  int32_t emission_dtype; /* FLTOP_EMISSION_*: element type of the emissions */
   int32_t device;         /* CUDA device ordinal */
   void* workspace;        /* optional DEVICE memory, 256-byte aligned, for all of the
                              handle's scratch; NULL = the library allocates it */
@@ -98,8 +109,9 @@ size_t fltop_workspace_size(const fltop_config* cfg);
 int fltop_create(const fltop_config* cfg, fltop_handle** out);
 
 /* Algorithm 1 for a whole batch.  Each of the B utterances is decoded independently.
- *   d_logp      [B,T,V] float32 log-probabilities; element strides stride_b, stride_t, the
- *               V entries of a frame contiguous and 16-byte aligned when V % 4 == 0.
+ *   d_logp      [B,T,V] log-probabilities (emission_dtype); element strides stride_b, stride_t,
+ *               the V entries of a frame contiguous.  Rows that start on a multiple of four
+ *               elements' bytes, with V % 4 == 0, take the fast path.
  *               Frames t >= d_lengths[b] are never read.
  *   d_lengths   [B] int32 frame counts.
  *   d_tokens    [B,K,L] int32: hypothesis k of utterance b, L = max_out_len; entries past
@@ -110,7 +122,7 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out);
  *   d_nhyp      [B] int32 number of hypotheses (<= K; 1 with the empty sequence and score 0
  *               when the length is 0).
  *   d_status    [B] int32 FLTOP_ST_* bits, may be NULL. */
-int fltop_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+int fltop_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t stride_t,
                  const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_tokens,
                  int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
                  void* cuda_stream);
@@ -118,7 +130,7 @@ int fltop_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t
 /* fltop_decode for callers whose emissions and results live in HOST memory (Algorithm 1 is
  * stated on host arrays; this is the same procedure with the transfers done by the library).
  * fltop_enable_host_io allocates, once, what that takes: device copies of the inputs and
- * outputs ([max_batch, max_frames, V] float32 + [max_batch, K, L] int32 + small arrays), a few
+ * outputs ([max_batch, max_frames, V] emissions + [max_batch, K, L] int32 + small arrays), a few
  * KB of pinned host memory, sixteen streams.  FLTOP_ERR_STATE on a streaming handle,
  * FLTOP_ERR_OOM / FLTOP_ERR_CUDA if an allocation fails (the handle stays usable for the
  * device-pointer calls); calling it again is a no-op. */
@@ -137,7 +149,7 @@ int fltop_enable_host_io(fltop_handle* h);
  * are busy at once; a process that leaves CUDA_DEVICE_MAX_CONNECTIONS at its default of 8 lets
  * them share hardware queues, which costs a few per cent.)  FLTOP_ERR_STATE unless
  * fltop_enable_host_io succeeded on this handle. */
-int fltop_decode_host(fltop_handle* h, const float* h_logp, int64_t stride_b, int64_t stride_t,
+int fltop_decode_host(fltop_handle* h, const void* h_logp, int64_t stride_b, int64_t stride_t,
                       const int32_t* h_lengths, int32_t B, int32_t T, int32_t* h_tokens,
                       int32_t* h_lens, float* h_scores, int32_t* h_nhyp, int32_t* h_status,
                       void* cuda_stream);
@@ -146,14 +158,14 @@ int fltop_last_host_io_bytes(const fltop_handle* h, int64_t* out);
 
 /* Algorithm 1 consumed chunk by chunk: the frame loop of S concurrent streams advances by
  * up to C frames; the beam of every stream is kept in the handle between calls.
- *   d_chunk      [S,C,V] float32, contiguous.
+ *   d_chunk      [S,C,V] emission_dtype, contiguous.
  *   d_chunk_lens [S] int32 valid frames of each stream in this chunk (0 = idle).
  *   d_flags      [S] uint8, may be NULL: bit0 = reset the stream to the empty prefix before
  *                consuming the chunk; bit1 = write this stream's current hypotheses.
  *                NULL means "no reset, write hypotheses if output pointers are given".
  *                A stream must be reset before its first chunk.
  *   outputs as in fltop_decode with B = S; all four may be NULL together (no readback). */
-int fltop_stream_step(fltop_handle* h, const float* d_chunk, const int32_t* d_chunk_lens,
+int fltop_stream_step(fltop_handle* h, const void* d_chunk, const int32_t* d_chunk_lens,
                       const uint8_t* d_flags, int32_t S, int32_t C, int32_t* d_tokens,
                       int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
                       void* cuda_stream);
@@ -166,7 +178,7 @@ int fltop_destroy(fltop_handle* h);
  *   d_counts  [B,T] int32 survivors per frame (0 for frames past the length).
  *   d_entries [B,T,V] pairs {int32 token, float32 logp}; the first d_counts[b,t] pairs of
  *             frame (b,t) are valid. */
-int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+int fltop_prune(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t stride_t,
                 const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_counts,
                 void* d_entries, void* cuda_stream);
 

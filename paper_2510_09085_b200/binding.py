@@ -33,8 +33,13 @@ class fltop_config(C.Structure):
                 ("threshold_r", C.c_float), ("max_batch", C.c_int32), ("max_frames", C.c_int32),
                 ("max_chunk_frames", C.c_int32), ("max_out_len", C.c_int32),
                 ("top_n", C.c_int32), ("beam_threshold", C.c_float), ("merge_max", C.c_int32),
-                ("device", C.c_int32),
+                ("emission_dtype", C.c_int32), ("device", C.c_int32),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+FLTOP_EMISSION_F32, FLTOP_EMISSION_F16, FLTOP_EMISSION_BF16 = 0, 1, 2
+EMISSION_CODES = {torch.float32: FLTOP_EMISSION_F32, torch.float16: FLTOP_EMISSION_F16,
+                  torch.bfloat16: FLTOP_EMISSION_BF16}
 
 
 class FltopError(RuntimeError):
@@ -105,10 +110,11 @@ def status_string(code: int) -> str:
 
 def make_config(vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                 max_chunk_frames=0, max_out_len=None, device=0, workspace=0, workspace_bytes=0,
-                top_n=0, beam_threshold=0.0, merge_max=0) -> fltop_config:
+                top_n=0, beam_threshold=0.0, merge_max=0, emission_dtype=0) -> fltop_config:
     return fltop_config(vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                         max_chunk_frames, max_frames if max_out_len is None else max_out_len,
-                        top_n, beam_threshold, int(merge_max), device, workspace or None,
+                        top_n, beam_threshold, int(merge_max), int(emission_dtype), device,
+                        workspace or None,
                         workspace_bytes)
 
 
@@ -174,10 +180,12 @@ class Decoder:
 
     def __init__(self, vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                  max_chunk_frames=0, max_out_len=None, device=0, top_n=0, beam_threshold=0.0,
-                 merge_max=False):
+                 merge_max=False, emission_dtype=torch.float32):
         self.cfg = make_config(vocab_size, blank_id, beam_width, threshold_r, max_batch,
                                max_frames, max_chunk_frames, max_out_len, device, top_n=top_n,
-                               beam_threshold=beam_threshold, merge_max=int(bool(merge_max)))
+                               beam_threshold=beam_threshold, merge_max=int(bool(merge_max)),
+                               emission_dtype=EMISSION_CODES[emission_dtype])
+        self.emission_dtype = emission_dtype
         code, self.h = fltop_create(self.cfg)
         if code != FLTOP_OK:
             self.h = None
@@ -192,8 +200,9 @@ class Decoder:
 
     # --- batch ---------------------------------------------------------------------
     def decode(self, logp: torch.Tensor, lengths: torch.Tensor, stream=None):
-        """logp [B,T,V] float32 CUDA (last dim contiguous), lengths [B] int32 CUDA."""
-        assert logp.is_cuda and logp.dtype == torch.float32 and logp.stride(2) == 1
+        """logp [B,T,V] CUDA of the handle's emission dtype (last dim contiguous), lengths [B]
+        int32 CUDA."""
+        assert logp.is_cuda and logp.dtype == self.emission_dtype and logp.stride(2) == 1
         assert lengths.is_cuda and lengths.dtype == torch.int32 and lengths.is_contiguous()
         B, T, _ = logp.shape
         code = fltop_decode(self.h, logp, logp.stride(0), logp.stride(1), lengths, B, T,
@@ -218,7 +227,7 @@ class Decoder:
     def decode_host(self, logp: torch.Tensor, lengths: torch.Tensor, stream=None):
         """logp [B,T,V] float32 and lengths [B] int32 in HOST memory; the results are in the
         host tensors h_tokens / h_lens / h_scores / h_nhyp / h_status when this returns."""
-        assert not logp.is_cuda and logp.dtype == torch.float32 and logp.stride(2) == 1
+        assert not logp.is_cuda and logp.dtype == self.emission_dtype and logp.stride(2) == 1
         assert not lengths.is_cuda and lengths.dtype == torch.int32 and lengths.is_contiguous()
         B, T, _ = logp.shape
         code = lib().fltop_decode_host(self.h, _p(logp), logp.stride(0), logp.stride(1),
@@ -247,7 +256,7 @@ class Decoder:
     # --- streaming -----------------------------------------------------------------
     def stream_step(self, chunk: torch.Tensor, chunk_lens: torch.Tensor, flags=None,
                     readback=True, stream=None):
-        assert chunk.is_cuda and chunk.dtype == torch.float32 and chunk.is_contiguous()
+        assert chunk.is_cuda and chunk.dtype == self.emission_dtype and chunk.is_contiguous()
         S, Cf, _ = chunk.shape
         outs = (self.tokens, self.lens, self.scores, self.nhyp) if readback else (None,) * 4
         code = fltop_stream_step(self.h, chunk, chunk_lens, flags, S, Cf, *outs, self.status,

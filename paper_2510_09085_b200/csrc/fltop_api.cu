@@ -21,7 +21,7 @@ struct HostIo {
   bool ready = false;
   unsigned char* dev = nullptr;      // one device allocation
   unsigned char* pinned = nullptr;   // one pinned host allocation
-  float* d_logp = nullptr;           // [max_batch, max_frames, V]
+  unsigned char* d_logp = nullptr;   // [max_batch, max_frames, V] elements of emission_dtype
   int32_t* d_lengths = nullptr;      // [max_batch]
   int32_t* d_tokens = nullptr;       // [max_batch, K, L]
   // lens [n,K], scores [n,K], nhyp [n], status [n] of a group of n utterances lie back to back
@@ -82,6 +82,7 @@ bool config_ok(const fltop_config* c) {
   if (c->top_n < 0) return false;
   if (c->beam_threshold != c->beam_threshold) return false;  // NaN
   if (c->merge_max != 0 && c->merge_max != 1) return false;
+  if (c->emission_dtype < FLTOP_EMISSION_F32 || c->emission_dtype > FLTOP_EMISSION_BF16) return false;
   if (c->device < 0) return false;
   if ((int64_t)(c->beam_width + 1) * c->max_frames + 2 > (int64_t)std::numeric_limits<int32_t>::max())
     return false;
@@ -136,7 +137,7 @@ struct DeviceGuard {
   }
 };
 
-int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t stride_t,
                const int32_t* d_lengths, const uint8_t* d_flags, int32_t B, int32_t T,
                bool streaming, int32_t* d_tokens, int32_t* d_lens, float* d_scores,
                int32_t* d_nhyp, int32_t* d_status, cudaStream_t s, int32_t slot0 = 0,
@@ -150,7 +151,8 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   if (B == 0) return FLTOP_OK;
 
   PruneParams pp;
-  pp.logp = d_logp; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
+  pp.logp = d_logp; pp.dtype = h->cfg.emission_dtype;
+  pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
   pp.counts = h->counts + (int64_t)slot0 * T;
   pp.entries = h->entries + (int64_t)slot0 * T * h->cfg.vocab_size;
@@ -164,8 +166,10 @@ int run_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t s
   dp.merge_max = h->cfg.merge_max;
   dp.counts = pp.counts; dp.entries = pp.entries;
   dp.nodes = h->nodes + (int64_t)slot0 * h->nodes_per_utt;
-  const bool fuse = h->fusion != 0 && T > 0 && decode_can_prune(h->cfg.vocab_size);
-  dp.logp = fuse ? d_logp : nullptr; dp.stride_b = stride_b; dp.stride_t = stride_t;
+  const bool fuse = h->fusion != 0 && T > 0 &&
+                    decode_can_prune(h->cfg.vocab_size, h->cfg.emission_dtype, d_logp, stride_b, stride_t);
+  dp.logp = fuse ? d_logp : nullptr; dp.dtype = h->cfg.emission_dtype;
+  dp.stride_b = stride_b; dp.stride_t = stride_t;
   dp.log_r = h->log_r;
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
@@ -227,7 +231,7 @@ int fltop_enable_host_io(fltop_handle* h) {
   const size_t L = (size_t)h->cfg.max_out_len;
   const size_t n_logp = B * (size_t)h->cfg.max_frames * (size_t)h->cfg.vocab_size;
   size_t off = 0;
-  const size_t o_logp = off; off += up(n_logp * 4);
+  const size_t o_logp = off; off += up(n_logp * emission_bytes(h->cfg.emission_dtype));
   const size_t o_len = off; off += up(B * 4);
   const size_t o_tok = off; off += up(B * K * L * 4);
   const size_t o_small = off; off += up(B * (2 * K + 2) * 4);
@@ -238,7 +242,7 @@ int fltop_enable_host_io(fltop_handle* h) {
     return e == cudaErrorMemoryAllocation ? FLTOP_ERR_OOM : cuda_fail(h, e);
   }
   io.dev = static_cast<unsigned char*>(ptr);
-  io.d_logp = reinterpret_cast<float*>(io.dev + o_logp);
+  io.d_logp = io.dev + o_logp;
   io.d_lengths = reinterpret_cast<int32_t*>(io.dev + o_len);
   io.d_tokens = reinterpret_cast<int32_t*>(io.dev + o_tok);
   io.d_small = reinterpret_cast<int32_t*>(io.dev + o_small);
@@ -268,7 +272,7 @@ int fltop_enable_host_io(fltop_handle* h) {
   return FLTOP_OK;
 }
 
-int fltop_decode_host(fltop_handle* h, const float* h_logp, int64_t stride_b, int64_t stride_t,
+int fltop_decode_host(fltop_handle* h, const void* h_logp, int64_t stride_b, int64_t stride_t,
                       const int32_t* h_lengths, int32_t B, int32_t T, int32_t* h_tokens,
                       int32_t* h_lens, float* h_scores, int32_t* h_nhyp, int32_t* h_status,
                       void* cuda_stream) {
@@ -319,6 +323,8 @@ int fltop_decode_host(fltop_handle* h, const float* h_logp, int64_t stride_b, in
 
   int rc = FLTOP_OK;
   const int64_t row_pitch = (int64_t)T * V;  // device staging: [slot, T, V], this call's T
+  const int64_t esize = (int64_t)emission_bytes(h->cfg.emission_dtype);
+  const unsigned char* const h_bytes = static_cast<const unsigned char*>(h_logp);
   for (int32_t gi = 0; gi < n_groups && rc == FLTOP_OK; ++gi) {
     const int32_t s0 = group_begin(gi), n = group_begin(gi + 1) - s0;
     cudaStream_t st = io.stream[gi];
@@ -329,19 +335,19 @@ int fltop_decode_host(fltop_handle* h, const float* h_logp, int64_t stride_b, in
       const int32_t u = io.order[slot];
       const int64_t len = usable(u);
       if (len == 0) continue;
-      float* dst = io.d_logp + (int64_t)slot * row_pitch;
-      const float* src = h_logp + (int64_t)u * stride_b;
+      unsigned char* dst = io.d_logp + (int64_t)slot * row_pitch * esize;
+      const unsigned char* src = h_bytes + (int64_t)u * stride_b * esize;
       if (stride_t == V) {
-        e = cudaMemcpyAsync(dst, src, (size_t)(len * V) * 4, cudaMemcpyHostToDevice, st);
+        e = cudaMemcpyAsync(dst, src, (size_t)(len * V * esize), cudaMemcpyHostToDevice, st);
       } else {
-        e = cudaMemcpy2DAsync(dst, (size_t)V * 4, src, (size_t)stride_t * 4, (size_t)V * 4,
-                              (size_t)len, cudaMemcpyHostToDevice, st);
+        e = cudaMemcpy2DAsync(dst, (size_t)(V * esize), src, (size_t)(stride_t * esize),
+                              (size_t)(V * esize), (size_t)len, cudaMemcpyHostToDevice, st);
       }
-      io.h2d_bytes += len * V * 4;
+      io.h2d_bytes += len * V * esize;
     }
     if (e != cudaSuccess) { rc = cuda_fail(h, e); break; }
     int32_t* const small = io.d_small + (int64_t)s0 * (2 * K + 2);
-    rc = run_decode(h, io.d_logp + (int64_t)s0 * row_pitch, row_pitch, V, io.d_lengths + s0,
+    rc = run_decode(h, io.d_logp + (int64_t)s0 * row_pitch * esize, row_pitch, V, io.d_lengths + s0,
                     nullptr, n, T, false, io.d_tokens + (int64_t)s0 * K * L, small,
                     reinterpret_cast<float*>(small + (int64_t)n * K), small + (int64_t)2 * n * K,
                     small + (int64_t)2 * n * K + n, st, s0, B);
@@ -481,7 +487,7 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   return FLTOP_OK;
 }
 
-int fltop_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+int fltop_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t stride_t,
                  const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_tokens,
                  int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
                  void* cuda_stream) {
@@ -497,7 +503,7 @@ int fltop_decode(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t
                     d_lens, d_scores, d_nhyp, d_status, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int fltop_stream_step(fltop_handle* h, const float* d_chunk, const int32_t* d_chunk_lens,
+int fltop_stream_step(fltop_handle* h, const void* d_chunk, const int32_t* d_chunk_lens,
                       const uint8_t* d_flags, int32_t S, int32_t C, int32_t* d_tokens,
                       int32_t* d_lens, float* d_scores, int32_t* d_nhyp, int32_t* d_status,
                       void* cuda_stream) {
@@ -514,7 +520,7 @@ int fltop_stream_step(fltop_handle* h, const float* d_chunk, const int32_t* d_ch
                     d_lens, d_scores, d_nhyp, d_status, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t stride_t,
+int fltop_prune(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t stride_t,
                 const int32_t* d_lengths, int32_t B, int32_t T, int32_t* d_counts,
                 void* d_entries, void* cuda_stream) {
   if (!h) return FLTOP_ERR_INVALID_ARG;
@@ -526,7 +532,8 @@ int fltop_prune(fltop_handle* h, const float* d_logp, int64_t stride_b, int64_t 
   cudaError_t e = g.enter(h->cfg.device);
   if (e != cudaSuccess) return cuda_fail(h, e);
   PruneParams pp;
-  pp.logp = d_logp; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
+  pp.logp = d_logp; pp.dtype = h->cfg.emission_dtype;
+  pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
   pp.counts = d_counts; pp.entries = static_cast<Survivor*>(d_entries);
   e = launch_prune(pp, static_cast<cudaStream_t>(cuda_stream));

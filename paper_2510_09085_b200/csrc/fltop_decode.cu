@@ -58,6 +58,9 @@
 //
 // Scores are float32 relative to a per-frame reference within a few nats of
 // the best total; the sum of the references is kept in float64.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "fltop_internal.h"
 
 namespace fltop {
@@ -584,13 +587,28 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   auto raw_row = [&](int t1) -> float* {
     return reinterpret_cast<float*>(smem) + (t1 & 3) * kFusedMaxV;
   };
+  // float32 rows: a word per lane; fp16 / bf16 rows: a word holds two tokens (V is even then)
   auto fetch_row = [&](int t1) {
-    if (lane < V)
-      cp_async4(raw_row(t1) + lane, p.logp + (int64_t)b * p.stride_b + (int64_t)t1 * p.stride_t + lane);
+    const int64_t at = (int64_t)b * p.stride_b + (int64_t)t1 * p.stride_t;
+    if (p.dtype == kEmissionF32) {
+      if (lane < V) cp_async4(raw_row(t1) + lane, static_cast<const float*>(p.logp) + at + lane);
+    } else if (2 * lane < V) {
+      cp_async4(raw_row(t1) + lane, static_cast<const uint16_t*>(p.logp) + at + 2 * lane);
+    }
   };
-  // the row of frame t1 has landed (each lane reads the word it fetched); returns the count
+  // the row of frame t1 has landed; returns the survivor count
   auto prune_row = [&](int t1) -> int {
-    const float v = lane < V ? raw_row(t1)[lane] : neg_inf();
+    float v = neg_inf();
+    if (p.dtype == kEmissionF32) {
+      if (lane < V) v = raw_row(t1)[lane];  // the word this lane fetched itself
+    } else {
+      __syncwarp();  // the word was fetched by lane / 2
+      if (lane < V) {
+        const unsigned short bits = reinterpret_cast<const unsigned short*>(raw_row(t1))[lane];
+        v = p.dtype == kEmissionF16 ? __half2float(__ushort_as_half(bits))
+                                    : __bfloat162float(__ushort_as_bfloat16(bits));
+      }
+    }
     // row maximum through an order-preserving integer key (a NaN never is the maximum)
     const unsigned vu = __float_as_uint(v);
     const unsigned vkey = (v == v) ? ((vu & 0x80000000u) ? ~vu : (vu | 0x80000000u)) : 0x007fffffu;
@@ -1337,7 +1355,13 @@ void launch_variant(const DecodeParams& p, int nt, size_t bytes, bool alone, cud
 }
 }  // namespace
 
-bool decode_can_prune(int V) { return V <= kFusedMaxV; }
+bool decode_can_prune(int V, int dtype, const void* logp, int64_t stride_b, int64_t stride_t) {
+  if (V > kFusedMaxV) return false;
+  if (dtype == kEmissionF32) return true;
+  // two-byte elements are fetched in pairs: every row has to start on a four-byte boundary
+  return V % 2 == 0 && stride_b % 2 == 0 && stride_t % 2 == 0 &&
+         (reinterpret_cast<uintptr_t>(logp) & 3u) == 0;
+}
 
 cudaError_t decode_prepare(int K, int V) {
   const int bytes = (int)decode_smem_bytes(K, V);

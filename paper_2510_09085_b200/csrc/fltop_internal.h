@@ -34,8 +34,14 @@ constexpr int kStateHeaderWords = sizeof(StateHeader) / 4;
 constexpr int kStateWordsPerSlot = 10;
 inline size_t state_words(int K) { return kStateHeaderWords + (size_t)kStateWordsPerSlot * K; }
 
+// How the emissions are stored (FLTOP_EMISSION_* of the public header); always widened to
+// float32 before anything is computed.
+enum { kEmissionF32 = 0, kEmissionF16 = 1, kEmissionBF16 = 2 };
+inline size_t emission_bytes(int dtype) { return dtype == kEmissionF32 ? 4 : 2; }
+
 struct PruneParams {
-  const float* logp;
+  const void* logp;         // elements of `dtype`
+  int32_t dtype;
   int64_t stride_b, stride_t;
   const int32_t* lengths;   // [B]
   int32_t B, T, V;
@@ -62,7 +68,8 @@ struct DecodeParams {
                             // each utterance's total in its first frame's place, zeros after)
   const Survivor* entries;  // [B*T*V]
   // Non-null: the decode kernel prunes the rows itself (V <= 32) and `entries` is not read.
-  const float* logp;
+  const void* logp;         // elements of `dtype`
+  int32_t dtype;
   int64_t stride_b, stride_t;
   float log_r;
   TrieNode* nodes;          // [B * nodes_per_utt]
@@ -83,6 +90,7 @@ cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
 cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s);
 cudaError_t decode_prepare(int K, int V);  // one-time kernel attribute set-up
-bool decode_can_prune(int V);            // the decode kernel can take raw emission rows
+// the decode kernel can take these raw emission rows itself (strides in elements)
+bool decode_can_prune(int V, int dtype, const void* logp, int64_t stride_b, int64_t stride_t);
 
 }  // namespace fltop

@@ -6,7 +6,12 @@
 // This is the one stage that streams the emissions from HBM.  A row is read
 // exactly once with 128-bit loads, kept in registers while the row maximum is
 // reduced with warp shuffles, and compacted with ballot + popc, so the kernel
-// moves 4*V bytes in and 8*S + 4 bytes out per frame.
+// moves 4*V bytes in and 8*S + 4 bytes out per frame.  Emissions stored as
+// fp16 or bf16 are widened to float32 on load (exact), so the comparison is
+// the same float32 comparison and the row costs 2*V bytes.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "fltop_internal.h"
 
 namespace fltop {
@@ -23,9 +28,29 @@ __device__ __forceinline__ bool row_is_live(const PruneParams& p, int64_t row, i
   return len <= p.T && t < len;  // a negative or oversized length reads nothing
 }
 
+// Four consecutive emissions, widened to float32: one 16-byte or 8-byte streaming load.
+__device__ __forceinline__ float4 load_quad(const float* src) {
+  return __ldcs(reinterpret_cast<const float4*>(src));
+}
+__device__ __forceinline__ float4 load_quad(const __half* src) {
+  const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(src));
+  const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+  const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+  return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ float4 load_quad(const __nv_bfloat16* src) {
+  const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(src));
+  const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+  const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+  return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ float load_one(const float* src) { return *src; }
+__device__ __forceinline__ float load_one(const __half* src) { return __half2float(*src); }
+__device__ __forceinline__ float load_one(const __nv_bfloat16* src) { return __bfloat162float(*src); }
+
 // LPR lanes cooperate on one row (LPR a power of two <= 32); every lane holds
-// CH float4: tokens 4*LPR*i + 4*sub + j for i < CH, j < 4.
-template <int LPR, int CH>
+// CH float4: tokens 4*LPR*i + 4*sub + j for i < CH, j < 4.  E: the stored element type.
+template <typename E, int LPR, int CH>
 __global__ void __launch_bounds__(kPruneThreads) prune_vec_kernel(PruneParams p) {
   constexpr int ROWS_PER_WARP = 32 / LPR;
   const int lane = threadIdx.x & 31;
@@ -44,12 +69,12 @@ __global__ void __launch_bounds__(kPruneThreads) prune_vec_kernel(PruneParams p)
     const bool live = row < n_rows && row_is_live(p, row, b, t);
     float4 x[CH];
     float m = neg_inf();
-    const float* src = p.logp + (int64_t)b * p.stride_b + (int64_t)t * p.stride_t;
+    const E* src = static_cast<const E*>(p.logp) + (int64_t)b * p.stride_b + (int64_t)t * p.stride_t;
 #pragma unroll
     for (int i = 0; i < CH; ++i) {
       const int tok0 = 4 * LPR * i + 4 * sub;
       if (live && tok0 < p.V) {
-        x[i] = __ldcs(reinterpret_cast<const float4*>(src + tok0));
+        x[i] = load_quad(src + tok0);
       } else {
         x[i] = make_float4(neg_inf(), neg_inf(), neg_inf(), neg_inf());
       }
@@ -94,6 +119,7 @@ __global__ void __launch_bounds__(kPruneThreads) prune_vec_kernel(PruneParams p)
 
 // Any V, any alignment: one warp per row, two passes over the row (the second
 // pass is served by L1/L2).
+template <typename E>
 __global__ void __launch_bounds__(kPruneThreads) prune_scalar_kernel(PruneParams p) {
   const int lane = threadIdx.x & 31;
   const int64_t n_rows = (int64_t)p.B * p.T;
@@ -106,9 +132,9 @@ __global__ void __launch_bounds__(kPruneThreads) prune_scalar_kernel(PruneParams
       if (lane == 0) p.counts[row] = 0;
       continue;
     }
-    const float* src = p.logp + (int64_t)b * p.stride_b + (int64_t)t * p.stride_t;
+    const E* src = static_cast<const E*>(p.logp) + (int64_t)b * p.stride_b + (int64_t)t * p.stride_t;
     float m = neg_inf();
-    for (int c = lane; c < p.V; c += 32) m = fmaxf(m, src[c]);
+    for (int c = lane; c < p.V; c += 32) m = fmaxf(m, load_one(src + c));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     const float thr = __fadd_rn(m, p.log_r);
@@ -116,7 +142,7 @@ __global__ void __launch_bounds__(kPruneThreads) prune_scalar_kernel(PruneParams
     int base = 0;
     for (int c0 = 0; c0 < p.V; c0 += 32) {
       const int c = c0 + lane;
-      const float v = c < p.V ? src[c] : neg_inf();
+      const float v = c < p.V ? load_one(src + c) : neg_inf();
       const bool k = c < p.V && v >= thr;
       const unsigned bal = __ballot_sync(0xffffffffu, k);
       if (k) dst[base + __popc(bal & ((1u << lane) - 1u))] = Survivor{c, v};
@@ -235,7 +261,7 @@ __global__ void __launch_bounds__(kPruneThreads) topn_cap_kernel(PruneParams p, 
   }
 }
 
-template <int LPR, int CH>
+template <typename E, int LPR, int CH>
 cudaError_t launch_vec(const PruneParams& p, cudaStream_t s, int sms) {
   const int64_t n_rows = (int64_t)p.B * p.T;
   const int rows_per_block = (kPruneThreads / 32) * (32 / LPR);
@@ -243,7 +269,35 @@ cudaError_t launch_vec(const PruneParams& p, cudaStream_t s, int sms) {
   const int64_t cap = (int64_t)sms * 8;  // 8 resident blocks of 256 threads per SM
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  prune_vec_kernel<LPR, CH><<<(unsigned)blocks, kPruneThreads, 0, s>>>(p);
+  prune_vec_kernel<E, LPR, CH><<<(unsigned)blocks, kPruneThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename E>
+cudaError_t launch_prune_typed(const PruneParams& p, cudaStream_t s) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  // four elements at a time: rows have to start on a multiple of four elements' bytes
+  const bool aligned = (p.V % 4 == 0) && (p.stride_b % 4 == 0) && (p.stride_t % 4 == 0) &&
+                       ((reinterpret_cast<uintptr_t>(p.logp) & (4 * sizeof(E) - 1)) == 0);
+  if (aligned) {
+    const int quads = p.V / 4;
+    if (quads <= 1) return launch_vec<E, 1, 1>(p, s, sms);
+    if (quads <= 2) return launch_vec<E, 2, 1>(p, s, sms);
+    if (quads <= 4) return launch_vec<E, 4, 1>(p, s, sms);
+    if (quads <= 8) return launch_vec<E, 8, 1>(p, s, sms);
+    if (quads <= 16) return launch_vec<E, 16, 1>(p, s, sms);
+    if (quads <= 32) return launch_vec<E, 32, 1>(p, s, sms);
+    if (quads <= 64) return launch_vec<E, 32, 2>(p, s, sms);
+    if (quads <= 128) return launch_vec<E, 32, 4>(p, s, sms);
+    if (quads <= 256) return launch_vec<E, 32, 8>(p, s, sms);
+    if (quads <= 512) return launch_vec<E, 32, 16>(p, s, sms);
+  }
+  const int64_t n_rows = (int64_t)p.B * p.T;
+  int64_t blocks = (n_rows + (kPruneThreads / 32) - 1) / (kPruneThreads / 32);
+  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+  prune_scalar_kernel<E><<<(unsigned)blocks, kPruneThreads, 0, s>>>(p);
   return cudaGetLastError();
 }
 
@@ -251,29 +305,11 @@ cudaError_t launch_vec(const PruneParams& p, cudaStream_t s, int sms) {
 
 cudaError_t launch_prune(const PruneParams& p, cudaStream_t s) {
   if ((int64_t)p.B * p.T == 0) return cudaSuccess;
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const bool aligned = (p.V % 4 == 0) && (p.stride_b % 4 == 0) && (p.stride_t % 4 == 0) &&
-                       ((reinterpret_cast<uintptr_t>(p.logp) & 15u) == 0);
-  if (aligned) {
-    const int quads = p.V / 4;
-    if (quads <= 1) return launch_vec<1, 1>(p, s, sms);
-    if (quads <= 2) return launch_vec<2, 1>(p, s, sms);
-    if (quads <= 4) return launch_vec<4, 1>(p, s, sms);
-    if (quads <= 8) return launch_vec<8, 1>(p, s, sms);
-    if (quads <= 16) return launch_vec<16, 1>(p, s, sms);
-    if (quads <= 32) return launch_vec<32, 1>(p, s, sms);
-    if (quads <= 64) return launch_vec<32, 2>(p, s, sms);
-    if (quads <= 128) return launch_vec<32, 4>(p, s, sms);
-    if (quads <= 256) return launch_vec<32, 8>(p, s, sms);
-    if (quads <= 512) return launch_vec<32, 16>(p, s, sms);
+  switch (p.dtype) {
+    case kEmissionF16: return launch_prune_typed<__half>(p, s);
+    case kEmissionBF16: return launch_prune_typed<__nv_bfloat16>(p, s);
+    default: return launch_prune_typed<float>(p, s);
   }
-  const int64_t n_rows = (int64_t)p.B * p.T;
-  int64_t blocks = (n_rows + (kPruneThreads / 32) - 1) / (kPruneThreads / 32);
-  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
-  prune_scalar_kernel<<<(unsigned)blocks, kPruneThreads, 0, s>>>(p);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s) {

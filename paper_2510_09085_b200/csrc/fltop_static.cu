@@ -84,7 +84,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   PruneParams pp;
-  pp.logp = d_logp; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
+  pp.logp = d_logp; pp.dtype = kEmissionF32; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = vocab_size;
   pp.log_r = threshold_r > 0.f ? (float)std::log((double)threshold_r)
                                : -std::numeric_limits<float>::infinity();
@@ -97,7 +97,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   dp.emit_default = 1; dp.block_threads = 0; dp.co_resident = 0; dp.pruning = threshold_r >= 5e-4f ? 1 : 0;
   dp.top_n = 0; dp.beam_threshold = 0.f; dp.merge_max = 0;
   dp.counts = pp.counts; dp.entries = pp.entries;
-  dp.logp = nullptr; dp.stride_b = 0; dp.stride_t = 0; dp.log_r = pp.log_r;
+  dp.logp = nullptr; dp.dtype = kEmissionF32; dp.stride_b = 0; dp.stride_t = 0; dp.log_r = pp.log_r;
   dp.nodes = reinterpret_cast<TrieNode*>(scratch + kCountsBytes + kEntriesBytes);
   dp.nodes_per_utt = nodes_per_utt; dp.state = nullptr;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;

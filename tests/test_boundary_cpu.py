@@ -40,7 +40,7 @@ def test_config_struct_matches_header(bd):
     dict(vocab_size=1), dict(vocab_size=9000), dict(blank_id=-1), dict(blank_id=32),
     dict(beam_width=0), dict(beam_width=5000), dict(threshold_r=-0.1), dict(threshold_r=1.5),
     dict(threshold_r=float("nan")), dict(max_batch=0), dict(max_frames=0), dict(max_out_len=0),
-    dict(top_n=-1), dict(beam_threshold=float("nan")), dict(merge_max=2), dict(device=-1), dict(max_chunk_frames=-1),
+    dict(top_n=-1), dict(beam_threshold=float("nan")), dict(merge_max=2), dict(emission_dtype=3), dict(emission_dtype=-1), dict(device=-1), dict(max_chunk_frames=-1),
     dict(max_chunk_frames=101), dict(workspace=8, workspace_bytes=1 << 40),
     dict(beam_width=2048, vocab_size=8192),     # needs more shared memory than one SM has
 ])
@@ -56,7 +56,7 @@ def test_invalid_config_is_rejected_on_the_host(bd, kw):
 
 def test_optional_knobs_of_algorithm_1_are_accepted(bd):
     for kw in (dict(top_n=4), dict(beam_threshold=25.0), dict(top_n=100, beam_threshold=-1.0),
-               dict(merge_max=1)):
+               dict(merge_max=1), dict(emission_dtype=1), dict(emission_dtype=2)):
         cfg = bd.make_config(32, 0, 8, 0.01, 4, 100, **kw)
         assert bd.fltop_workspace_size(cfg) > 0
 
