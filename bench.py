@@ -42,18 +42,19 @@ NODE_BYTES, SURVIVOR_BYTES = 8, 8
 DECODE_DRAM_BYTES = 7.40e6
 
 
-def _algorithmic_bytes(V, st, out_bytes, fused):
+def _algorithmic_bytes(V, st, out_bytes, fused, esize=4):
     """(prune kernel, decode kernel) HBM bytes that one call has to move.
 
     Two kernels: the prune kernel reads every emission row and writes a count and the survivor
     list per frame, the decode kernel reads those back.  One kernel (it prunes its own rows):
     the emission rows are the decode kernel's input and no survivor list exists.  Either way
     the decode kernel writes one block of 8-byte trie records per frame (one record per beam
-    slot, rounded up to an even count) and the hypotheses at the end."""
+    slot, rounded up to an even count) and the hypotheses at the end.  ``esize``: bytes per
+    stored emission (4, or 2 for fp16 / bf16)."""
     trie = NODE_BYTES * (st["live_hypotheses_sum"] + st["frames"])
     if fused:
-        return 0, st["frames"] * 4 * V + trie + out_bytes
-    prune = st["frames"] * (4 * V + 4) + st["survivors"] * SURVIVOR_BYTES
+        return 0, st["frames"] * esize * V + trie + out_bytes
+    prune = st["frames"] * (esize * V + 4) + st["survivors"] * SURVIVOR_BYTES
     return prune, st["frames"] * 4 + st["survivors"] * SURVIVOR_BYTES + trie + out_bytes
 
 
@@ -384,18 +385,21 @@ def run_report(args):
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     rows = []
 
-    def measure(wl, K, r, label, top1_ref=None, top_n=0, theta=0.0):
+    def measure(wl, K, r, label, top1_ref=None, top_n=0, theta=0.0, merge_max=False,
+                dtype=torch.float32):
         B, T, V = wl.emissions.shape
-        x = torch.from_numpy(wl.emissions).cuda()
+        x = torch.from_numpy(wl.emissions).cuda().to(dtype)
         ln = torch.from_numpy(wl.lengths).cuda()
-        dec = binding.Decoder(V, wl.blank_id, K, r, B, T, top_n=top_n, beam_threshold=theta)
+        dec = binding.Decoder(V, wl.blank_id, K, r, B, T, top_n=top_n, beam_threshold=theta,
+                              merge_max=merge_max, emission_dtype=dtype)
         dec.set_profiling(True)
         ms, pk, dk = _time_decode(dec, x, ln, flush)
         st = dec.last_call_stats()
         assert int((dec.status != 0).sum()) == 0
         frames = int(wl.lengths.sum())
         pbytes, dbytes = _algorithmic_bytes(
-            V, st, 4 * int(dec.lens.sum()) + 8 * int(dec.nhyp.sum()) + 8 * B, fused=(pk == 0.0))
+            V, st, 4 * int(dec.lens.sum()) + 8 * int(dec.nhyp.sum()) + 8 * B, fused=(pk == 0.0),
+            esize=x.element_size())
         agree = None
         if top1_ref is not None:
             agree = sum(dec.hyps(b)[0][0] == top1_ref[b] for b in range(B)) / B
@@ -435,6 +439,11 @@ def run_report(args):
     sub = workloads.workload_subword()
     for r in sub.thresholds:
         measure(sub, sub.beam_width, r, "3 subword")
+    # variants: best-alignment scores (merge by max) and emissions stored in half precision
+    measure(wav, wav.beam_width, R_PRUNED, "V wav2vec2, merge by max", merge_max=True)
+    measure(wav, wav.beam_width, R_PRUNED, "V wav2vec2, fp16 emissions", dtype=torch.float16)
+    measure(sub, sub.beam_width, R_PRUNED, "V subword, fp16 emissions", dtype=torch.float16)
+    measure(sub, sub.beam_width, R_PRUNED, "V subword, bf16 emissions", dtype=torch.bfloat16)
     # streaming: 1024 streams, 16-frame chunks, beam state carried in the handle
     stw = workloads.workload_streaming()
     S, T, V = stw.emissions.shape
