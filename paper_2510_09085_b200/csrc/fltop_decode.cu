@@ -205,6 +205,13 @@ __host__ __device__ inline int table_size(int K) {
   while (n < want) n <<= 1;
   return n;
 }
+// log(exp(a) + exp(b) + exp(c)): one pass, the three exponentials independent of one another.
+__device__ __forceinline__ float lse3(float a, float b, float c) {
+  const float hi = fmaxf(fmaxf(a, b), c);
+  if (hi == neg_inf()) return hi;
+  return hi + __logf(__expf(a - hi) + __expf(b - hi) + __expf(c - hi));
+}
+
 constexpr unsigned kEmptySlot = 0xffffffffu;  // table entry: [tag : 20][beam slot : 12]
 // words of the bitmap over a frame's extension candidates (at most K * V of them)
 __host__ __device__ inline int dup_words(int K, int V) { return (K * ((V + 31) / 32) + 3) & ~3; }
@@ -722,16 +729,15 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     auto stay_eval = [&](int q) -> float {
       const Hot e = hc[q];
       const float npb = e.tot + fi.lp_blank;
-      float npnb = neg_inf();
+      float own = neg_inf(), dup = neg_inf();  // non-blank mass: the entry's own, its parent's
       if (e.last >= 0) {
         const float le = lpv[e.last];
-        npnb = e.pnb + le;
+        own = e.pnb + le;
         const int pq = table_find(tab_c, id_c, id_c[q].pprint);
         if (pq >= 0) {
           const Hot pe = hc[pq];
-          const float dup = ((pe.last == e.last) ? pe.pb : pe.tot) + le;
+          dup = ((pe.last == e.last) ? pe.pb : pe.tot) + le;
           if (dup != neg_inf()) {  // the parent's extension by last(q) names this prefix
-            npnb = use_max ? fmaxf(npnb, dup) : lse2(npnb, dup);
             atomicSub(&hist[score_bin(dup)], 1u);
             const int jp = jpos[e.last];  // position among all survivors -> among non-blank
             const int ed = pq * Snb + jp - ((blank_j >= 0 && jp > blank_j) ? 1 : 0);
@@ -739,10 +745,12 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           }
         }
       }
+      // masses are summed, or (merge_max) the better one is taken.  The total is formed from
+      // the three terms directly, not from npnb: the two results do not wait for each other.
+      const float npnb = use_max ? fmaxf(own, dup) : lse2(own, dup);
+      const float tot = use_max ? fmaxf(npb, fmaxf(own, dup)) : lse3(npb, own, dup);
       st_pb[q] = npb;
       st_pnb[q] = npnb;
-      // a prefix' blank and non-blank mass: summed, or (merge_max) the better one
-      const float tot = use_max ? fmaxf(npb, npnb) : lse2(npb, npnb);
       st_tot[q] = tot;
       if (tot != neg_inf()) count(tot);
       return tot;
