@@ -108,3 +108,16 @@ def test_host_calls_are_refused_where_they_cannot_work():
     with pytest.raises(b.FltopError):
         s.enable_host_io()
     s.close()
+
+
+def test_host_buffers_on_the_benchmark_batch():
+    # the full wav2vec2-shaped batch (B=64, K=50, r=1e-3) as bench.py's end-to-end leg runs it
+    wl = W.workload_wav2vec2()
+    B = wl.emissions.shape[0]
+    d = _both(wl.emissions, wl.lengths, 32, 50, 1e-3)
+    assert (d.h_status[:B] == 0).all()
+    _check_same(d, B)
+    h2d, d2h = d.host_io_bytes()
+    assert h2d == 4 * B + 4 * 32 * int(wl.lengths.sum())
+    assert d2h < 0.3 * d.tokens.numel() * 4          # far less than the padded token tensor
+    d.close()
