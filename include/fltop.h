@@ -241,6 +241,14 @@ int fltop_set_block_threads(fltop_handle* h, int32_t threads);
  * wider vocabularies take the separate prune kernel.  mode 0: always the separate kernel.
  * Results do not depend on it.  FLTOP_ERR_INVALID_ARG for a null handle or another mode. */
 int fltop_set_fusion(fltop_handle* h, int mode);
+/* Which decode kernel serves narrow problems (beam_width <= 32, vocab_size <= 32, pruning
+ * inside the kernel, no beam_threshold, no merge_max, no block size set).  The library has two:
+ * one thread block per utterance, and one warp per utterance with several utterances to a block.
+ * A warp alone is slower on its utterance but an SM runs many more of them side by side.
+ * mode 1 (the default): the warp kernel when a call brings at least eight utterances or streams
+ * per SM; mode 0: never; mode 2: whenever the problem is narrow enough.  Results are the same up
+ * to the order of exactly tied hypotheses.  FLTOP_ERR_INVALID_ARG for another mode. */
+int fltop_set_warp_decode(fltop_handle* h, int mode);
 int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
 
 #ifdef __cplusplus

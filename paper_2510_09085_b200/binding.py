@@ -25,7 +25,7 @@ EXPORTS = ("fltop_workspace_size", "fltop_create", "fltop_decode", "fltop_stream
            "fltop_beam_state_bytes", "fltop_launch_count", "fltop_last_call_stats", "fltop_set_profiling",
            "fltop_last_kernel_ms", "fltop_decode_static", "fltop_set_block_threads",
            "fltop_set_fusion", "fltop_enable_host_io", "fltop_decode_host",
-           "fltop_last_host_io_bytes")
+           "fltop_last_host_io_bytes", "fltop_set_warp_decode")
 
 
 class fltop_config(C.Structure):
@@ -91,6 +91,8 @@ def lib():
         L.fltop_set_block_threads.argtypes = [vp, i32]
         L.fltop_set_fusion.restype = C.c_int
         L.fltop_set_fusion.argtypes = [vp, C.c_int]
+        L.fltop_set_warp_decode.restype = C.c_int
+        L.fltop_set_warp_decode.argtypes = [vp, C.c_int]
         L.fltop_enable_host_io.restype = C.c_int
         L.fltop_enable_host_io.argtypes = [vp]
         L.fltop_decode_host.restype = C.c_int
@@ -299,6 +301,11 @@ class Decoder:
         code = lib().fltop_set_fusion(self.h, int(mode))
         if code != FLTOP_OK:
             raise FltopError(code, "fltop_set_fusion")
+
+    def set_warp_decode(self, mode: int):
+        code = lib().fltop_set_warp_decode(self.h, int(mode))
+        if code != FLTOP_OK:
+            raise FltopError(code, "fltop_set_warp_decode")
 
     def last_kernel_ms(self):
         ms = (C.c_float * 2)()

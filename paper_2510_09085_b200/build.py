@@ -8,8 +8,9 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libfltop.so")
-SOURCES = ["fltop_api.cu", "fltop_prune.cu", "fltop_decode.cu", "fltop_static.cu"]
-HEADERS = [os.path.join(CSRC, "fltop_internal.h"),
+SOURCES = ["fltop_api.cu", "fltop_prune.cu", "fltop_decode.cu", "fltop_decode_warp.cu",
+           "fltop_static.cu"]
+HEADERS = [os.path.join(CSRC, "fltop_internal.h"), os.path.join(CSRC, "fltop_device.cuh"),
            os.path.join(os.path.dirname(PKG), "include", "fltop.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--extended-lambda", "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]

@@ -59,6 +59,7 @@ struct fltop_handle {
   int64_t launches;
   int32_t block_threads;  // 0 = chosen by the library
   int32_t fusion;         // 1 = the decode kernel prunes where it can
+  int32_t warp_mode;      // warp-per-utterance kernel: 0 never, 1 when it pays, 2 whenever it can
   bool profiling;
   bool prof_valid;
   cudaEvent_t ev[3];
@@ -161,7 +162,7 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
   dp.lengths = d_lengths; dp.flags = d_flags; dp.B = B; dp.T = T; dp.V = h->cfg.vocab_size;
   dp.K = h->cfg.beam_width; dp.blank = h->cfg.blank_id; dp.L = h->cfg.max_out_len;
   dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
-  dp.block_threads = h->block_threads; dp.co_resident = co_resident; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
+  dp.block_threads = h->block_threads; dp.warp_mode = h->warp_mode; dp.co_resident = co_resident; dp.pruning = h->cfg.threshold_r >= 5e-4f ? 1 : 0;  // weaker thresholds keep most tokens
   dp.top_n = h->cfg.top_n; dp.beam_threshold = h->cfg.beam_threshold;
   dp.merge_max = h->cfg.merge_max;
   dp.counts = pp.counts; dp.entries = pp.entries;
@@ -191,7 +192,7 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
     }
   }
   if (timed) cudaEventRecord(h->ev[1], s);
-  e = launch_decode(dp, s);
+  e = decode_warp_eligible(dp) ? launch_decode_warp(dp, s) : launch_decode(dp, s);
   if (e != cudaSuccess) return cuda_fail(h, e);
   ++h->launches;
   if (timed) {
@@ -447,6 +448,7 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   h->last_cuda = 0; h->launches = 0; h->profiling = false; h->prof_valid = false;
   h->block_threads = 0;
   h->fusion = 1;
+  h->warp_mode = 1;
   h->ev[0] = h->ev[1] = h->ev[2] = nullptr;
   if (cfg->workspace) {
     h->ws = static_cast<unsigned char*>(cfg->workspace);
@@ -607,6 +609,12 @@ int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
 int fltop_set_fusion(fltop_handle* h, int mode) {
   if (!h || (mode != 0 && mode != 1)) return FLTOP_ERR_INVALID_ARG;
   h->fusion = mode;
+  return FLTOP_OK;
+}
+
+int fltop_set_warp_decode(fltop_handle* h, int mode) {
+  if (!h || mode < 0 || mode > 2) return FLTOP_ERR_INVALID_ARG;
+  h->warp_mode = mode;
   return FLTOP_OK;
 }
 

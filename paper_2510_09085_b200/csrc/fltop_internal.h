@@ -57,6 +57,7 @@ struct DecodeParams {
   int32_t streaming;        // 0: reset at entry, no state kept.  1: state loaded / stored
   int32_t emit_default;     // streaming with flags == null: emit results?
   int32_t block_threads;    // 0 = choose from K, V and whether pruning is on
+  int32_t warp_mode;        // warp-per-utterance kernel: 0 never, 1 when it pays, 2 whenever it can
   int32_t co_resident;      // utterance blocks on the GPU at the same time as this launch's,
                             // its own included (0 = just its own B): launches of one batch
                             // split over several streams size their blocks for the whole batch
@@ -89,6 +90,9 @@ cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
 // keeps at most top_n survivors per frame (no-op for top_n <= 0 or >= V)
 cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s);
+// narrow beams over narrow vocabularies: one warp per utterance (fltop_decode_warp.cu)
+bool decode_warp_eligible(const DecodeParams& p);
+cudaError_t launch_decode_warp(const DecodeParams& p, cudaStream_t s);
 cudaError_t decode_prepare(int K, int V);  // one-time kernel attribute set-up
 // the decode kernel can take these raw emission rows itself (strides in elements)
 bool decode_can_prune(int V, int dtype, const void* logp, int64_t stride_b, int64_t stride_t);

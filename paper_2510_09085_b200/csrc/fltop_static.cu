@@ -94,7 +94,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   DecodeParams dp;
   dp.lengths = d_lengths; dp.flags = nullptr; dp.B = B; dp.T = T; dp.V = vocab_size;
   dp.K = beam_width; dp.blank = blank_id; dp.L = max_out_len; dp.streaming = 0;
-  dp.emit_default = 1; dp.block_threads = 0; dp.co_resident = 0; dp.pruning = threshold_r >= 5e-4f ? 1 : 0;
+  dp.emit_default = 1; dp.block_threads = 0; dp.co_resident = 0; dp.warp_mode = 0; dp.pruning = threshold_r >= 5e-4f ? 1 : 0;
   dp.top_n = 0; dp.beam_threshold = 0.f; dp.merge_max = 0;
   dp.counts = pp.counts; dp.entries = pp.entries;
   dp.logp = nullptr; dp.dtype = kEmissionF32; dp.stride_b = 0; dp.stride_t = 0; dp.log_r = pp.log_r;
