@@ -476,6 +476,35 @@ def run_report(args):
                   "beam_state_bytes": dec.beam_state_bytes}
     print(json.dumps(stream_row), file=sys.stderr, flush=True)
     dec.close()
+
+    # many more streams than SMs: chunks queued back to back, device time, with the decode kernel
+    # the library picks by itself (one warp per stream) and with the block-per-stream kernel
+    def many_streams(streams, mode):
+        w = workloads.workload_streaming(streams=streams, chunks=8)
+        S2, T2, _ = w.emissions.shape
+        x2 = torch.from_numpy(w.emissions).cuda()
+        d2 = binding.Decoder(V, 0, K, r, S2, T2, max_chunk_frames=C)
+        d2.set_warp_decode(mode)
+        full2 = torch.full((S2,), C, dtype=torch.int32, device="cuda")
+        n2 = T2 // C
+        ch = [x2[:, i * C:(i + 1) * C].contiguous() for i in range(n2)]
+        fl = [torch.full((S2,), (1 if i == 0 else 0) | (2 if i == n2 - 1 else 0), dtype=torch.uint8,
+                         device="cuda") for i in range(n2)]
+        best = None
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(True), torch.cuda.Event(True)
+            e0.record()
+            for i in range(n2):
+                d2.stream_step(ch[i], full2, fl[i], readback=(i == n2 - 1))
+            e1.record()
+            e1.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None or ms < best else best
+        assert int((d2.status != 0).sum()) == 0
+        d2.close()
+        return {"streams": S2, "frames_per_s": S2 * T2 / (best * 1e-3), "us_per_chunk": 1e3 * best / n2}
+    many = [(many_streams(n_s, 1), many_streams(n_s, 0)) for n_s in (4096, 16384)]
+    print(json.dumps(many), file=sys.stderr, flush=True)
     # CPU oracle, single thread, on a sample of the wav2vec2 workload (a reported baseline)
     order = np.argsort(wav.lengths)
     sample = [int(i) for i in order[::8]]
@@ -499,6 +528,12 @@ def run_report(args):
                 f"{stream_row['frames_per_s']:.3g} frames/s aggregate, chunk latency p50 "
                 f"{stream_row['p50_ms']:.3f} ms, p99 {stream_row['p99_ms']:.3f} ms (host wall clock, "
                 f"call to stream sync), beam state {stream_row['beam_state_bytes'] / 1e6:.1f} MB.\n")
+        for auto, block in many:
+            f.write(f"\nStreaming, {auto['streams']} streams (same K, r, chunks of {C} frames queued back to "
+                    f"back, device time): {auto['frames_per_s']:.3g} frames/s, {auto['us_per_chunk']:.0f} us "
+                    f"per chunk with the warp-per-stream kernel the library picks at this size; "
+                    f"{block['frames_per_s']:.3g} frames/s, {block['us_per_chunk']:.0f} us with the "
+                    f"block-per-stream kernel.\n")
         f.write(f"\nCPU oracle, one thread, 8 of the 64 wav2vec2 utterances, K=50: "
                 f"{cpu_p:.0f} frames/s at r=1e-3, {cpu_0:.0f} frames/s at r=0.\n")
 
