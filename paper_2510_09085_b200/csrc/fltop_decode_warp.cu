@@ -124,11 +124,11 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
   };
   // Table of the beam's fingerprints: entries [tag : 20 | slot : 12], linear probing, never
   // more than a quarter full.
-  auto rebuild_table = [&](const BeamCopy& c, int n) {
+  auto rebuild_table = [&](int n) {  // from the fingerprints in the registers
     reinterpret_cast<uint4*>(S.tab)[lane] = make_uint4(kFree, kFree, kFree, kFree);
     __syncwarp();
     if (lane < n) {
-      const unsigned long long h = c.print[lane];
+      const unsigned long long h = e_print;
       const unsigned val = (((unsigned)h & 0xfffffu) << 12) | (unsigned)lane;
       unsigned pos = (unsigned)(h >> 40) & (kWarpTab - 1);
       while (atomicCAS(&S.tab[pos], kFree, val) != kFree) pos = (pos + 1) & (kWarpTab - 1);
@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
   publish_beam(S.beam[cur]);
   clear_frame_scratch();
   __syncwarp();
-  rebuild_table(S.beam[cur], nb);
+  rebuild_table(nb);
   __syncwarp();
 
   const int64_t row0 = (int64_t)b * p.stride_b;
@@ -266,6 +266,30 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       }
     };
 
+    // the same for the lane that owns the source entry: everything is in its registers
+    auto place_own_stay = [&](int slot) {
+      N.last[slot] = e_last;
+      N.pb[slot] = npb - best;
+      N.pnb[slot] = npnb - best;
+      N.tot[slot] = stot - best;
+      N.print[slot] = e_print;
+      N.pprint[slot] = e_pprint;
+      N.node[slot] = e_node;
+      N.len[slot] = e_len;
+    };
+    auto place_own_ext = [&](int c, float sc, int slot) {
+      N.last[slot] = c;
+      N.pb[slot] = neg_inf();
+      N.pnb[slot] = sc - best;
+      N.tot[slot] = sc - best;
+      N.print[slot] = child_print(e_print, c);
+      N.pprint[slot] = e_print;
+      N.node[slot] = arena_ok ? n_nodes + slot : 0;
+      N.len[slot] = e_len + 1;
+      if (arena_ok) nodes[n_nodes + slot] = TrieNode{e_node, c};
+      ++created;
+    };
+
     if (take_all || cut.cut_count <= kListCap) {
       // the cut as scores (bin edges): > f_hi is above the cut bin, > f_lo in it or above
       const float f_lo = (cut.thr >= kFastBins - 1) ? neg_inf()
@@ -278,7 +302,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       const bool s_sure = stot > f_hi, s_list = !s_sure && stot > f_lo;
       const unsigned bs = __ballot_sync(kFull, s_sure);
       const int n_stay = __popc(bs);
-      if (s_sure) place(lane, 0, stot, __popc(bs & lt_mask));
+      if (s_sure) place_own_stay(__popc(bs & lt_mask));
       {
         const unsigned bl = __ballot_sync(kFull, s_list);
         if (s_list) {
@@ -295,7 +319,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
         if ((my_dup >> c) & 1u) sc = neg_inf();  // merged into a stay candidate
         const bool x_sure = sc > f_hi, x_list = !x_sure && sc > f_lo;
         const unsigned bx = __ballot_sync(kFull, x_sure);
-        if (x_sure) place(lane, c + 1, sc, nbn - 1 - (n_ext + __popc(bx & lt_mask)));
+        if (x_sure) place_own_ext(c, sc, nbn - 1 - (n_ext + __popc(bx & lt_mask)));
         n_ext += __popc(bx);
         const unsigned bl = __ballot_sync(kFull, x_list);
         if (x_list) {
@@ -353,10 +377,10 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       {
         const bool above = s_key > kth, tie = s_key == kth && kth != 0u;
         const unsigned ba = __ballot_sync(kFull, above);
-        if (above) place(lane, 0, stot, __popc(ba & lt_mask));
+        if (above) place_own_stay(__popc(ba & lt_mask));
         const unsigned bt = __ballot_sync(kFull, tie);
         const int r = __popc(bt & lt_mask);
-        if (tie && r < need) place(lane, 0, stot, n_above_stay + r);
+        if (tie && r < need) place_own_stay(n_above_stay + r);
         n_tie += min(__popc(bt), need);
       }
       for (unsigned m = kb; m; m &= m - 1) {
@@ -366,11 +390,11 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
         const unsigned key = score_key(sc);
         const bool above = key > kth, tie = key == kth && kth != 0u;
         const unsigned ba = __ballot_sync(kFull, above);
-        if (above) place(lane, c + 1, sc, nbn - 1 - (n_ext + __popc(ba & lt_mask)));
+        if (above) place_own_ext(c, sc, nbn - 1 - (n_ext + __popc(ba & lt_mask)));
         n_ext += __popc(ba);
         const unsigned bt = __ballot_sync(kFull, tie);
         const int r = n_tie + __popc(bt & lt_mask);
-        if (tie && r < need) place(lane, c + 1, sc, n_above_stay + r);
+        if (tie && r < need) place_own_ext(c, sc, n_above_stay + r);
         n_tie = min(n_tie + __popc(bt), need);
       }
     }
@@ -392,7 +416,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
     nb = nbn;
     cur ^= 1;
     clear_frame_scratch();
-    rebuild_table(S.beam[cur], nb);
+    rebuild_table(nb);
     __syncwarp();
   }
   frames_seen += len;
