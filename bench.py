@@ -273,8 +273,8 @@ def run_ours(args):
     dk_ms = statistics.mean(decode_p)
     achieved = db / (dk_ms * 1e-3) / 1e9
     h2d, d2h = dec_p.host_io_bytes()  # counted by the library from the copies it issued
-    e2e_same = all(torch.equal(d.cpu(), h) for d, h in ((dec_p.lens, dec_p.h_lens),
-                                                        (dec_p.scores, dec_p.h_scores),
+    # (scores and counts only: which of two exactly tied hypotheses comes first is not unique)
+    e2e_same = all(torch.equal(d.cpu(), h) for d, h in ((dec_p.scores, dec_p.h_scores),
                                                         (dec_p.nhyp, dec_p.h_nhyp)))
     assert e2e_same, "host-buffer decode and device-buffer decode disagree"
 
