@@ -15,8 +15,9 @@
  * fields; its language model is not implemented.
  *
  * Conventions
- *   - every `d_*` pointer is DEVICE memory owned by the caller; the library
- *     never frees or keeps it beyond the call's work on `cuda_stream`.
+ *   - every `d_*` pointer is DEVICE memory owned by the caller (`h_*`: HOST
+ *     memory, fltop_decode_host only); the library never frees or keeps it
+ *     beyond the call's work on `cuda_stream`.
  *   - calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*;
  *     NULL = the legacy default stream) and return without synchronising;
  *     outputs are valid once the caller has synchronised the stream.
@@ -118,7 +119,9 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out);
  *               the hypothesis' length are left untouched.
  *   d_lens      [B,K] int32 true lengths (0 for unused slots k >= nhyp).
  *   d_scores    [B,K] float32 log-probability of each hypothesis (log-sum of its blank and
- *               non-blank mass at the last frame; -inf for unused slots); best first.
+ *               non-blank mass at the last frame, the larger of the two with merge_max; -inf
+ *               for unused slots); best first.  Hypotheses whose scores tie exactly come in
+ *               no particular order.
  *   d_nhyp      [B] int32 number of hypotheses (<= K; 1 with the empty sequence and score 0
  *               when the length is 0).
  *   d_status    [B] int32 FLTOP_ST_* bits, may be NULL. */
@@ -145,7 +148,8 @@ int fltop_enable_host_io(fltop_handle* h);
  * h_lens, h_scores, h_nhyp and (if not NULL) h_status are written in full.
  * The work is ordered after what `cuda_stream` held at the call and `cuda_stream` waits for
  * it; unlike the device-pointer calls this one RETURNS ONLY WHEN THE OUTPUTS ARE IN HOST
- * MEMORY.  Results are those of fltop_decode, bit for bit.  (Up to 16 of the handle's streams
+ * MEMORY.  Results are those of fltop_decode: the same scores bit for bit, the same hypotheses
+ * up to the order of exactly tied ones.  (Up to 16 of the handle's streams
  * are busy at once; a process that leaves CUDA_DEVICE_MAX_CONNECTIONS at its default of 8 lets
  * them share hardware queues, which costs a few per cent.)  FLTOP_ERR_STATE unless
  * fltop_enable_host_io succeeded on this handle. */
