@@ -909,7 +909,26 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           list_id[li] = id;
         }
       };
-      if (is_stay) {
+      if (is_stay && NS <= 64 && !kWide) {
+        // At most two stay warps: each looks at all (at most 64) stay candidates itself, so the
+        // places follow from two ballots and no counter is shared.
+        const float s_lo = lane < nb ? st_tot[lane] : neg_inf();
+        const float s_hi = 32 + lane < nb ? st_tot[32 + lane] : neg_inf();
+        const int k_lo = klass(s_lo), k_hi = klass(s_hi);
+        const unsigned m_lo = __ballot_sync(kFull, k_lo == 2);
+        const unsigned m_hi = __ballot_sync(kFull, k_hi == 2);
+        const bool upper = warp != 0;
+        const float sc = upper ? s_hi : s_lo;
+        const int kl = upper ? k_hi : k_lo;
+        // a stay lane has no use for the extension-score registers: they carry its own
+        // candidate and the slot it won over the barrier, and it writes it to the next beam itself
+        int at = -1;
+        if (kl == 2) at = upper ? __popc(m_lo) + __popc(m_hi & lt_mask) : __popc(m_lo & lt_mask);
+        kc[0] = sc;
+        kc[1] = __int_as_float(at < K ? at : -1);
+        if (tid == 0) sc_c[SC_SLOT] = __popc(m_lo) + __popc(m_hi);  // read after B3
+        if (kl == 1) list_add(score_key(sc), tid << 16);
+      } else if (is_stay) {
         // stays are dense: one ballot per round, the warp's places taken by its first lane
         for (int base = 0; base < nb; base += NS) {
           const int i = base + tid;
@@ -981,7 +1000,10 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       // ranks the members of the cut bin exactly (score, then candidate id) and writes the
       // winners to the slots between the stays and the extensions.
       const int n_stay = min(sc_c[SC_SLOT], K);
-      if (is_stay) {
+      if (is_stay && NS <= 64 && !kWide) {
+        const int slot = __float_as_int(kc[1]);
+        if (slot >= 0) place_stay(tid, score_key(kc[0]), slot);
+      } else if (is_stay) {
         for (int s2 = tid; s2 < n_stay; s2 += NS) place_stay(sel_id[s2] >> 16, sel_key[s2], s2);
       } else if (is_ext) {
         const int n_ext = min(sc_c[SC_SLOT_E], K);
