@@ -156,6 +156,8 @@ __host__ __device__ inline int node_stage_len(int K) { return (K + 1) & ~1; }
 // Byte offsets of the shared-memory arrays.
 // widest vocabulary whose frames the decode block prunes itself (one token per lane)
 constexpr int kFusedMaxV = 32;
+// up to this many stay lanes, every stay warp looks at all stay candidates itself (P3a)
+constexpr int kOwnStayLanes = 128;
 
 struct Lay {
   unsigned sv, hot, ident, where, nstage, finfo, warp_sums, st_pb, st_pnb, st_tot, dup, tab, lpv,
@@ -909,24 +911,32 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           list_id[li] = id;
         }
       };
-      if (is_stay && NS <= 64 && !kWide) {
-        // At most two stay warps: each looks at all (at most 64) stay candidates itself, so the
-        // places follow from two ballots and no counter is shared.
-        const float s_lo = lane < nb ? st_tot[lane] : neg_inf();
-        const float s_hi = 32 + lane < nb ? st_tot[32 + lane] : neg_inf();
-        const int k_lo = klass(s_lo), k_hi = klass(s_hi);
-        const unsigned m_lo = __ballot_sync(kFull, k_lo == 2);
-        const unsigned m_hi = __ballot_sync(kFull, k_hi == 2);
-        const bool upper = warp != 0;
-        const float sc = upper ? s_hi : s_lo;
-        const int kl = upper ? k_hi : k_lo;
+      if (is_stay && NS <= kOwnStayLanes && !kWide) {
+        // At most four stay warps: each looks at all (at most 128) stay candidates itself, so
+        // the places follow from ballots alone and no counter is shared.
+        int before = 0, total_sel = 0;  // selected stays in the warps below this one / in all
+        float sc = neg_inf();
+        int kl = 0;
+        unsigned m_own = 0u;
+#pragma unroll
+        for (int w = 0; w < kOwnStayLanes / 32; ++w) {
+          if (w * 32 < NS) {
+            const float s_w = w * 32 + lane < nb ? st_tot[w * 32 + lane] : neg_inf();
+            const int k_w = klass(s_w);
+            const unsigned m_w = __ballot_sync(kFull, k_w == 2);
+            const int n_w = __popc(m_w);
+            before += w < warp ? n_w : 0;
+            total_sel += n_w;
+            if (w == warp) { sc = s_w; kl = k_w; m_own = m_w; }
+          }
+        }
         // a stay lane has no use for the extension-score registers: they carry its own
         // candidate and the slot it won over the barrier, and it writes it to the next beam itself
         int at = -1;
-        if (kl == 2) at = upper ? __popc(m_lo) + __popc(m_hi & lt_mask) : __popc(m_lo & lt_mask);
+        if (kl == 2) at = before + __popc(m_own & lt_mask);
         kc[0] = sc;
         kc[1] = __int_as_float(at < K ? at : -1);
-        if (tid == 0) sc_c[SC_SLOT] = __popc(m_lo) + __popc(m_hi);  // read after B3
+        if (tid == 0) sc_c[SC_SLOT] = total_sel;  // read after B3
         if (kl == 1) list_add(score_key(sc), tid << 16);
       } else if (is_stay) {
         // stays are dense: one ballot per round, the warp's places taken by its first lane
@@ -1000,7 +1010,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       // ranks the members of the cut bin exactly (score, then candidate id) and writes the
       // winners to the slots between the stays and the extensions.
       const int n_stay = min(sc_c[SC_SLOT], K);
-      if (is_stay && NS <= 64 && !kWide) {
+      if (is_stay && NS <= kOwnStayLanes && !kWide) {
         const int slot = __float_as_int(kc[1]);
         if (slot >= 0) place_stay(tid, score_key(kc[0]), slot);
       } else if (is_stay) {
