@@ -1181,7 +1181,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       if (n > Lout) truncated = true;
       int32_t* dst = p.out_tokens + o * Lout;
       int node = w.node;
-      for (int d = n - 1; d >= 0 && node > 0; --d) {
+      for (int d = n - 1; d >= 0 && node > 0 && (int64_t)node < p.nodes_per_utt; --d) {
         const int2 rec = *reinterpret_cast<const int2*>(&nodes[node]);  // parent, token
         if (d < Lout) dst[d] = rec.y;
         node = rec.x;

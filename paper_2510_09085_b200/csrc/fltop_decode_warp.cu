@@ -241,6 +241,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
     // Writing a candidate into slot `slot` of the next beam: q = 0 stays as it is, q > 0
     // (token + 1) is a new prefix and gets its trie record.
     auto place = [&](int q, int c_plus1, float sc, int slot) {
+      if ((unsigned)slot >= (unsigned)K) return;  // only reachable with NaN scores
       if (c_plus1 == 0) {
         N.last[slot] = C.last[q];
         N.pb[slot] = S.st_pb[q] - best;
@@ -268,6 +269,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
 
     // the same for the lane that owns the source entry: everything is in its registers
     auto place_own_stay = [&](int slot) {
+      if ((unsigned)slot >= (unsigned)K) return;
       N.last[slot] = e_last;
       N.pb[slot] = npb - best;
       N.pnb[slot] = npnb - best;
@@ -278,6 +280,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       N.len[slot] = e_len;
     };
     auto place_own_ext = [&](int c, float sc, int slot) {
+      if ((unsigned)slot >= (unsigned)K) return;
       N.last[slot] = c;
       N.pb[slot] = neg_inf();
       N.pnb[slot] = sc - best;
@@ -471,7 +474,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       if (e_len > Lout) truncated = true;
       int32_t* dst = p.out_tokens + o * Lout;
       int node = e_node;
-      for (int d = e_len - 1; d >= 0 && node > 0; --d) {
+      for (int d = e_len - 1; d >= 0 && node > 0 && (int64_t)node < p.nodes_per_utt; --d) {
         const int2 rec = *reinterpret_cast<const int2*>(&nodes[node]);  // parent, token
         if (d < Lout) dst[d] = rec.y;
         node = rec.x;
