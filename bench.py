@@ -39,7 +39,7 @@ L2_FLUSH_BYTES = 256 << 20
 NODE_BYTES, SURVIVOR_BYTES = 8, 8
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch on the default workload
 # (profiles/decode_kernel_wav2vec2_B64_K50_full.txt); None whenever the kernel has changed since
-DECODE_DRAM_BYTES = 8.11e6
+DECODE_DRAM_BYTES = 7.47e6
 
 
 def _algorithmic_bytes(V, st, out_bytes, fused, esize=4):
