@@ -114,13 +114,31 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def _workload(rank: int, args=None):
-    """The headline workload (wav2vec2-shaped, B=64, K=50) unless --workload / --batch say otherwise."""
-    from paper_2510_09085_b200 import workloads
-    if args is not None and args.workload == "subword":
-        return workloads.workload_subword(seed=2 + 1000 * rank, batch=args.batch or 256)
-    batch = (args.batch if args is not None and args.batch else BATCH)
-    return workloads.workload_wav2vec2(seed=1 + 1000 * rank, batch=batch, beam_width=BEAM)
+def _workload(rank: int, world: int = 1, args=None):
+    """This rank's share of the job's workload, and the number of utterances of the whole job.
+
+    The job decodes ONE batch of 64 utterances per GPU (wav2vec2-shaped, K=50, unless --workload
+    / --batch say otherwise).  It is split over the ranks by total frames, longest utterance
+    first (paper_2510_09085_b200/sharding.py); no data crosses ranks.  With --independent
+    every rank draws a batch of its own instead."""
+    import dataclasses
+    from paper_2510_09085_b200 import sharding, workloads
+    subword = args is not None and args.workload == "subword"
+    per_gpu = (args.batch if args is not None and args.batch else (256 if subword else BATCH))
+    independent = args is not None and args.independent
+
+    def draw(seed, batch):
+        if subword:
+            return workloads.workload_subword(seed=seed, batch=batch)
+        return workloads.workload_wav2vec2(seed=seed, batch=batch, beam_width=BEAM)
+    if world == 1 or independent:
+        return draw((2 if subword else 1) + 1000 * rank, per_gpu), per_gpu * world
+    whole = draw(2 if subword else 1, per_gpu * world)
+    mine = sharding.shard_of_rank(whole.lengths, rank, world)
+    T = max(1, int(whole.lengths[mine].max())) if len(mine) else 1
+    part = dataclasses.replace(whole, emissions=np.ascontiguousarray(whole.emissions[mine, :T]),
+                               lengths=np.ascontiguousarray(whole.lengths[mine]))
+    return part, per_gpu * world
 
 
 def _oracle_frames_per_s(wl, r, utterances):
@@ -138,7 +156,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = _workload(0)
+    wl, _ = _workload(0)
     order = np.argsort(wl.lengths)
     sample = [int(i) for i in order[::8]]          # 8 utterances spread over the length range
     for _ in range(args.warmup):
@@ -197,7 +215,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    wl = _workload(rank, args)
+    wl, n_global = _workload(rank, world, args)
     BEAM = wl.beam_width
     B, T, V = wl.emissions.shape
     n_frames = int(wl.lengths.sum())
@@ -548,6 +566,9 @@ def main():
     ap.add_argument("--workload", choices=["wav2vec2", "subword"], default="wav2vec2",
                     help="default: the headline wav2vec2-shaped batch; subword: V=1024, K=32")
     ap.add_argument("--batch", type=int, default=0, help="utterances per GPU (0 = the workload's own)")
+    ap.add_argument("--independent", action="store_true",
+                    help="N > 1: every rank draws a batch of its own instead of taking its share "
+                         "of one batch of N x 64 utterances")
     ap.add_argument("--report", metavar="FILE", help="measure all five workloads, write a table")
     ap.add_argument("--skip-oracle", action="store_true", help="--report without top-1 agreement")
     args = ap.parse_args()

@@ -116,7 +116,10 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out);
  *               Frames t >= d_lengths[b] are never read.
  *   d_lengths   [B] int32 frame counts.
  *   d_tokens    [B,K,L] int32: hypothesis k of utterance b, L = max_out_len; entries past
- *               the hypothesis' length are left untouched.
+ *               the hypothesis' length are left untouched.  Inside the search a prefix is
+ *               identified by a 64-bit fingerprint of its token sequence: two different
+ *               prefixes that are in the beam of the same frame and share all 64 bits would be
+ *               taken for one (chance about 2^-64 per pair and frame; not detected).
  *   d_lens      [B,K] int32 true lengths (0 for unused slots k >= nhyp).
  *   d_scores    [B,K] float32 log-probability of each hypothesis (log-sum of its blank and
  *               non-blank mass at the last frame, the larger of the two with merge_max; -inf
@@ -227,9 +230,13 @@ int fltop_last_cuda_error(const fltop_handle* h);
 size_t fltop_beam_state_bytes(const fltop_handle* h);
 /* Kernels launched by this handle since creation. */
 int64_t fltop_launch_count(const fltop_handle* h);
-/* Totals of the most recent decode / stream_step call (synchronises its stream):
+/* Totals of the most recent decode / stream_step call (synchronises its stream), eight values:
  * out[0] frames decoded, out[1] survivors over those frames, out[2] prefix-trie nodes
- * created, out[3] beam entries summed over frames (mean live hypotheses = out[3]/out[0]). */
+ * created, out[3] beam entries summed over frames (mean live hypotheses = out[3]/out[0]),
+ * out[4] the largest number of trie node ids any one utterance has used so far, out[5] probes
+ * of the fingerprint table that met a different prefix with the same 20-bit tag (each was
+ * told apart by the full 64 bits), out[6] frames whose selection took the slow exact path,
+ * out[7] reserved (0). */
 int fltop_last_call_stats(fltop_handle* h, int64_t* out);
 /* With profiling enabled every call brackets its kernels with CUDA events on the caller's
  * stream.  fltop_last_kernel_ms synchronises on those events and returns the device time
@@ -254,6 +261,31 @@ int fltop_set_fusion(fltop_handle* h, int mode);
  * to the order of exactly tied hypotheses.  FLTOP_ERR_INVALID_ARG for another mode. */
 int fltop_set_warp_decode(fltop_handle* h, int mode);
 int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
+
+/* Instrumented launches, for tests and profiling; everything is off on a new handle and no
+ * ordinary launch pays for it.  The paper has no counterpart.
+ *   FLTOP_HOOK_SURVIVOR_MASKS  d_buffer: DEVICE uint32 [B*T] of the next calls (NULL = off).
+ *       A decode kernel that prunes the frames itself (vocab_size <= 32) writes the survivor
+ *       set of frame (b,t) - bit c set iff token c survives Algorithm 1's top-N stage and
+ *       conditional break - to d_buffer[b*T + t]; frames past the length are left untouched.
+ *   FLTOP_HOOK_PHASE_CLOCKS    d_buffer: DEVICE int64 [b][32][8] (NULL = off): for frames
+ *       a <= t < a + b of utterance 0 the row kernel records the SM clock of every warp at its
+ *       eight phase boundaries (frame start, end of evaluation, after the first barrier, after
+ *       the histogram scan, end of placement, after the list barrier, before and after the
+ *       last barrier).
+ *   FLTOP_HOOK_TABLE_SLOTS     a: 0 (off) or a power of two: the shared-memory table of prefix
+ *       fingerprints is cut down to that many slots.  With fewer slots than beam entries its
+ *       bounded probe walks run out, which the kernels report as FLTOP_ST_INTERNAL.
+ *   FLTOP_HOOK_ROW_KERNEL      a: 1 (default) character vocabularies with beams of at most 64
+ *       take the row kernel; 0: they take the general block kernel.
+ * FLTOP_ERR_INVALID_ARG for a null handle, an unknown hook or a value out of range. */
+enum {
+  FLTOP_HOOK_SURVIVOR_MASKS = 1,
+  FLTOP_HOOK_PHASE_CLOCKS = 2,
+  FLTOP_HOOK_TABLE_SLOTS = 3,
+  FLTOP_HOOK_ROW_KERNEL = 4
+};
+int fltop_set_test_hook(fltop_handle* h, int hook, void* d_buffer, int64_t a, int64_t b);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,7 @@ EXPORTS = ("fltop_workspace_size", "fltop_create", "fltop_decode", "fltop_stream
            "fltop_beam_state_bytes", "fltop_launch_count", "fltop_last_call_stats", "fltop_set_profiling",
            "fltop_last_kernel_ms", "fltop_decode_static", "fltop_set_block_threads",
            "fltop_set_fusion", "fltop_enable_host_io", "fltop_decode_host",
-           "fltop_last_host_io_bytes", "fltop_set_warp_decode")
+           "fltop_last_host_io_bytes", "fltop_set_warp_decode", "fltop_set_test_hook")
 
 
 class fltop_config(C.Structure):
@@ -38,6 +38,8 @@ class fltop_config(C.Structure):
 
 
 FLTOP_EMISSION_F32, FLTOP_EMISSION_F16, FLTOP_EMISSION_BF16 = 0, 1, 2
+FLTOP_HOOK_SURVIVOR_MASKS, FLTOP_HOOK_PHASE_CLOCKS, FLTOP_HOOK_TABLE_SLOTS, \
+    FLTOP_HOOK_ROW_KERNEL = 1, 2, 3, 4
 EMISSION_CODES = {torch.float32: FLTOP_EMISSION_F32, torch.float16: FLTOP_EMISSION_F16,
                   torch.bfloat16: FLTOP_EMISSION_BF16}
 
@@ -99,6 +101,8 @@ def lib():
         L.fltop_decode_host.argtypes = [vp, vp, i64, i64, vp, i32, i32, vp, vp, vp, vp, vp, vp]
         L.fltop_last_host_io_bytes.restype = C.c_int
         L.fltop_last_host_io_bytes.argtypes = [vp, C.POINTER(C.c_int64)]
+        L.fltop_set_test_hook.restype = C.c_int
+        L.fltop_set_test_hook.argtypes = [vp, C.c_int, vp, i64, i64]
         L.fltop_decode_static.restype = C.c_int
         L.fltop_decode_static.argtypes = [i32, i32, i32, C.c_float, vp, i64, i64, vp, i32, i32,
                                           i32, vp, vp, vp, vp, vp, vp]
@@ -314,13 +318,20 @@ class Decoder:
             raise FltopError(code, "fltop_last_kernel_ms")
         return float(ms[0]), float(ms[1])
 
+    def set_test_hook(self, hook: int, buffer=None, a: int = 0, b: int = 0):
+        """fltop_set_test_hook; `buffer` is a CUDA tensor (kept alive by the caller) or None."""
+        code = lib().fltop_set_test_hook(self.h, int(hook), _p(buffer), int(a), int(b))
+        if code != FLTOP_OK:
+            raise FltopError(code, "fltop_set_test_hook")
+
     def last_call_stats(self) -> dict:
-        out = (C.c_int64 * 4)()
+        out = (C.c_int64 * 8)()
         code = lib().fltop_last_call_stats(self.h, out)
         if code != FLTOP_OK:
             raise FltopError(code, "fltop_last_call_stats")
         return {"frames": out[0], "survivors": out[1], "trie_nodes_created": out[2],
-                "live_hypotheses_sum": out[3]}
+                "live_hypotheses_sum": out[3], "max_node_ids_used": out[4],
+                "tag_clashes": out[5], "exact_select_frames": out[6]}
 
     @property
     def beam_state_bytes(self) -> int:

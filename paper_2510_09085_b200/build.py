@@ -8,7 +8,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libfltop.so")
-SOURCES = ["fltop_api.cu", "fltop_prune.cu", "fltop_decode.cu", "fltop_decode_warp.cu",
+SOURCES = ["fltop_api.cu", "fltop_prune.cu", "fltop_decode.cu", "fltop_decode_warp.cu", "fltop_decode_rows.cu",
            "fltop_static.cu"]
 HEADERS = [os.path.join(CSRC, "fltop_internal.h"), os.path.join(CSRC, "fltop_device.cuh"),
            os.path.join(os.path.dirname(PKG), "include", "fltop.h")]

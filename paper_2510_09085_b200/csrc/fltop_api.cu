@@ -60,9 +60,14 @@ struct fltop_handle {
   int32_t block_threads;  // 0 = chosen by the library
   int32_t fusion;         // 1 = the decode kernel prunes where it can
   int32_t warp_mode;      // warp-per-utterance kernel: 0 never, 1 when it pays, 2 whenever it can
+  int32_t rows_mode;      // 1: character vocabularies with beams up to 64 take the row kernel
   bool profiling;
   bool prof_valid;
   cudaEvent_t ev[3];
+  // instrumented launches (fltop_set_test_hook); all off by default
+  uint32_t* hook_masks;
+  long long* hook_clocks;
+  int32_t hook_frame0, hook_frames, hook_table_slots;
 };
 
 namespace {
@@ -110,7 +115,7 @@ Layout layout_of(const fltop_config& c) {
   l.state = off;
   if (c.max_chunk_frames > 0) off += up((size_t)c.max_batch * state_words(c.beam_width) * 4);
   l.beam_state = off;  // survivor lists + trie arenas + stream states
-  l.stats = off; off += up((size_t)c.max_batch * 4 * sizeof(int32_t));
+  l.stats = off; off += up((size_t)c.max_batch * kStatWords * sizeof(int32_t));
   l.total = off;  // survivor lists + trie arenas + stream states
   return l;
 }
@@ -158,7 +163,7 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
   pp.counts = h->counts + (int64_t)slot0 * T;
   pp.entries = h->entries + (int64_t)slot0 * T * h->cfg.vocab_size;
 
-  DecodeParams dp;
+  DecodeParams dp = {};
   dp.lengths = d_lengths; dp.flags = d_flags; dp.B = B; dp.T = T; dp.V = h->cfg.vocab_size;
   dp.K = h->cfg.beam_width; dp.blank = h->cfg.blank_id; dp.L = h->cfg.max_out_len;
   dp.streaming = streaming ? 1 : 0; dp.emit_default = 1;
@@ -175,7 +180,11 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
   dp.nodes_per_utt = h->nodes_per_utt; dp.state = h->state;
   dp.out_tokens = d_tokens; dp.out_lens = d_lens; dp.out_scores = d_scores; dp.out_nhyp = d_nhyp;
   dp.out_status = d_status;
-  dp.stats = h->stats + (int64_t)slot0 * 4;
+  dp.stats = h->stats + (int64_t)slot0 * kStatWords;
+  dp.table_slots = h->hook_table_slots;
+  dp.dbg_masks = h->hook_masks ? h->hook_masks + (int64_t)slot0 * T : nullptr;
+  dp.dbg_clocks = slot0 == 0 ? h->hook_clocks : nullptr;
+  dp.dbg_frame0 = h->hook_frame0; dp.dbg_frames = h->hook_frames;
   if (slot0 == 0) { h->last_B = B; h->last_T = T; h->last_stream = s; h->last_fused = fuse; }
 
   // (a batch decoded group by group on several streams is not timed kernel by kernel)
@@ -192,7 +201,9 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
     }
   }
   if (timed) cudaEventRecord(h->ev[1], s);
-  e = decode_warp_eligible(dp) ? launch_decode_warp(dp, s) : launch_decode(dp, s);
+  if (decode_warp_eligible(dp)) e = launch_decode_warp(dp, s);
+  else if (decode_rows_eligible(dp) && h->rows_mode != 0) e = launch_decode_rows(dp, s);
+  else e = launch_decode(dp, s);
   if (e != cudaSuccess) return cuda_fail(h, e);
   ++h->launches;
   if (timed) {
@@ -449,6 +460,9 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   h->block_threads = 0;
   h->fusion = 1;
   h->warp_mode = 1;
+  h->rows_mode = 1;
+  h->hook_masks = nullptr; h->hook_clocks = nullptr;
+  h->hook_frame0 = h->hook_frames = h->hook_table_slots = 0;
   h->ev[0] = h->ev[1] = h->ev[2] = nullptr;
   if (cfg->workspace) {
     h->ws = static_cast<unsigned char*>(cfg->workspace);
@@ -581,29 +595,59 @@ int64_t fltop_launch_count(const fltop_handle* h) { return h ? h->launches : 0; 
 
 int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
   if (!h || !out) return FLTOP_ERR_INVALID_ARG;
-  out[0] = out[1] = out[2] = out[3] = 0;
+  for (int i = 0; i < 8; ++i) out[i] = 0;
   if (h->last_B == 0) return FLTOP_OK;
   DeviceGuard g;
   cudaError_t e = g.enter(h->cfg.device);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->last_stream);
   if (e != cudaSuccess) return cuda_fail(h, e);
   const size_t B = (size_t)h->last_B, n_frames = B * (size_t)h->last_T;
-  int32_t* host = new (std::nothrow) int32_t[4 * B + n_frames];
+  int32_t* host = new (std::nothrow) int32_t[kStatWords * B + n_frames];
   if (!host) return FLTOP_ERR_OOM;
-  e = cudaMemcpy(host, h->stats, 4 * B * sizeof(int32_t), cudaMemcpyDeviceToHost);
+  e = cudaMemcpy(host, h->stats, kStatWords * B * sizeof(int32_t), cudaMemcpyDeviceToHost);
   if (e == cudaSuccess && n_frames)
-    e = cudaMemcpy(host + 4 * B, h->counts, n_frames * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    e = cudaMemcpy(host + kStatWords * B, h->counts, n_frames * sizeof(int32_t),
+                   cudaMemcpyDeviceToHost);
   if (e == cudaSuccess) {
     for (size_t b = 0; b < B; ++b) {
-      out[0] += host[4 * b];
-      out[2] += host[4 * b + 1];
-      out[3] += host[4 * b + 2];
+      const int32_t* s = host + kStatWords * b;
+      out[0] += s[0];
+      out[2] += s[1];
+      out[3] += s[2];
+      out[4] = std::max<int64_t>(out[4], s[3]);
+      out[5] += s[4];
+      out[6] += s[5];
     }
-    for (size_t i = 0; i < n_frames; ++i) out[1] += host[4 * B + i];
+    for (size_t i = 0; i < n_frames; ++i) out[1] += host[kStatWords * B + i];
   }
   delete[] host;
   if (e != cudaSuccess) return cuda_fail(h, e);
   return FLTOP_OK;
+}
+
+int fltop_set_test_hook(fltop_handle* h, int hook, void* d_buffer, int64_t a, int64_t b) {
+  if (!h) return FLTOP_ERR_INVALID_ARG;
+  switch (hook) {
+    case FLTOP_HOOK_SURVIVOR_MASKS:
+      h->hook_masks = static_cast<uint32_t*>(d_buffer);
+      return FLTOP_OK;
+    case FLTOP_HOOK_PHASE_CLOCKS:
+      if (d_buffer && (a < 0 || b < 1 || b > (1 << 20))) return FLTOP_ERR_INVALID_ARG;
+      h->hook_clocks = static_cast<long long*>(d_buffer);
+      h->hook_frame0 = (int32_t)a;
+      h->hook_frames = d_buffer ? (int32_t)b : 0;
+      return FLTOP_OK;
+    case FLTOP_HOOK_TABLE_SLOTS:
+      if (a < 0 || a > (1 << 20) || (a & (a - 1)) != 0) return FLTOP_ERR_INVALID_ARG;
+      h->hook_table_slots = (int32_t)a;
+      return FLTOP_OK;
+    case FLTOP_HOOK_ROW_KERNEL:
+      if (a != 0 && a != 1) return FLTOP_ERR_INVALID_ARG;
+      h->rows_mode = (int32_t)a;
+      return FLTOP_OK;
+    default:
+      return FLTOP_ERR_INVALID_ARG;
+  }
 }
 
 int fltop_set_fusion(fltop_handle* h, int mode) {

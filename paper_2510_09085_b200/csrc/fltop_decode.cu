@@ -135,7 +135,7 @@ enum {
   SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_MAXKEY, SC_PER_FRAME,
   // single copies
   SC_THR = 2 * SC_PER_FRAME, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_TOTAL, SC_FIRST, SC_STATUS,
-  SC_CREATED, SC_DEAD, SC_NLIVE, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL, SC_KEPT,
+  SC_CREATED, SC_CLASHES, SC_DEAD, SC_NLIVE, SC_MADE, SC_MADE_ODD, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL, SC_KEPT,
   // exact fallback select
   SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_NBEAM_NEXT, SC_COUNT
 };
@@ -297,7 +297,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   constexpr bool kWide = KMAX < 0;
   const int VS = VMAX > 0 ? VMAX : V;
   const Lay L = make_layout(KS, VS);
-  const int TS = table_size(KS);
+  // (a caller may shrink the table: only the test of the bounded probe walks does)
+  const int TS = p.table_slots > 0 ? min(p.table_slots, table_size(KS)) : table_size(KS);
   const int DW = dup_words(KS, VS);
   const int NSL = node_stage_len(KS);
   const unsigned tmask = (unsigned)TS - 1u;
@@ -365,7 +366,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   for (int i = tid; i < 2 * VS; i += NT) lpv_base[i] = neg_inf();
   for (int i = tid; i < 2 * kFastBins; i += NT) hist_base[i] = 0u;
   if (tid < SC_COUNT) scal[tid] = tid == SC_NEXT_BJ ? -1 : 0;
-  int created = 0, live_sum = 0;
+  int created = 0, live_sum = 0, tag_clashes = 0;
   int cur = 0, nb, n_nodes, frames_seen;
   double offset;
   if (do_reset) {
@@ -402,26 +403,34 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
 
   // Hash table of the beam's fingerprints.  An entry holds a beam slot and 20 bits of its
   // fingerprint, so a probe that meets another prefix is rejected without a second load; a
-  // tag match is confirmed against the full fingerprint.  The table is never more than half
-  // full, so a probe sequence always ends at an empty entry.
+  // tag match is confirmed against the full fingerprint.  The table is at most half full, so a
+  // probe sequence ends at an empty entry long before it has gone round; should it ever go
+  // round (TS probes), the walk gives up and the utterance is flagged FLTOP_ST_INTERNAL.
   auto table_insert = [&](unsigned* tab, unsigned long long h, int slot) {
     const unsigned val = (((unsigned)h & 0xfffffu) << 12) | (unsigned)slot;
     unsigned pos = (unsigned)(h >> 40) & tmask;
-    while (atomicCAS(&tab[pos], kEmptySlot, val) != kEmptySlot) pos = (pos + 1) & tmask;
+    for (int probes = 0; probes < TS; ++probes) {
+      if (atomicCAS(&tab[pos], kEmptySlot, val) == kEmptySlot) return;
+      pos = (pos + 1) & tmask;
+    }
+    atomicOr(&scal[SC_STATUS], 16);  // FLTOP_ST_INTERNAL: the entry is not in the table
   };
   // Beam slot of the entry with fingerprint h, or -1.
   auto table_find = [&](const unsigned* tab, const Ident* ids, unsigned long long h) {
     const unsigned tag = (unsigned)h & 0xfffffu;
     unsigned pos = (unsigned)(h >> 40) & tmask;
-    while (true) {
+    for (int probes = 0; probes < TS; ++probes) {
       const unsigned v = tab[pos];
       if (v == kEmptySlot) return -1;
       if ((v >> 12) == tag) {
         const int slot = (int)(v & 0xfffu);
         if (ids[slot].print == h) return slot;
+        ++tag_clashes;  // same 20-bit tag, another sequence
       }
       pos = (pos + 1) & tmask;
     }
+    atomicOr(&scal[SC_STATUS], 16);  // FLTOP_ST_INTERNAL
+    return -1;
   };
 
   const int32_t* counts = p.counts + (int64_t)b * p.T;
@@ -522,7 +531,10 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     }
     if ((kept >> lane) & 1u) svbuf(t1)[__popc(kept & lt_mask)] = Survivor{lane, v};
     const int n = __popc(kept);
-    if (lane == 0) scal[SC_KEPT] += n;  // survivors over all frames of this call
+    if (lane == 0) {
+      scal[SC_KEPT] += n;  // survivors over all frames of this call
+      if (p.dbg_masks) p.dbg_masks[(int64_t)b * p.T + t1] = kept;  // instrumented launches only
+    }
     return n;
   };
 
@@ -810,7 +822,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       atomicAdd(&scal[SC_DEAD], 1);
     };
     TrieNode* const nst = nstage + par * NSL;
-    // the frame's nodes get ids n_nodes .. n_nodes + nbn - 1 (the slots of stays stay unused)
+    // the frame's new prefixes get the node ids n_nodes, n_nodes + 1, ...
     const bool arena_ok = (int64_t)n_nodes + ((K + 1) & ~1) <= p.nodes_per_utt;
 
     // ---- P3: selected candidates take their slots in the next beam ---------------------
@@ -828,8 +840,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       wh_n[slot] = wh_c[q];
       table_insert(tab_n, id.print, slot);
     };
-    auto place_ext = [&](int q, int tok, unsigned key, int slot) {
-      if ((unsigned)slot >= (unsigned)K) return;
+    // a new prefix; `ord` numbers the frame's new prefixes (its trie record and node id)
+    auto place_ext = [&](int q, int tok, unsigned key, int slot, int ord) {
+      if ((unsigned)slot >= (unsigned)K || (unsigned)ord >= (unsigned)K) return;
       if (use_bt && key_score(key) < f_floor) return place_dead(slot);
       const float sc = key_score(key) - best;
       Hot e;
@@ -841,16 +854,16 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       table_insert(tab_n, h, slot);
       const Where w = wh_c[q];
       // back-pointer node: staged here, written to the trie in one piece after the frame
-      nst[slot] = TrieNode{w.node, tok};
+      nst[ord] = TrieNode{w.node, tok};
       ++created;
-      wh_n[slot] = Where{arena_ok ? n_nodes + slot : 0, w.len + 1};
+      wh_n[slot] = Where{arena_ok ? n_nodes + ord : 0, w.len + 1};
     };
     // a candidate by its id: beam entry in the high half, 0 (stay) or j + 1 (extension by the
     // j-th non-blank survivor) in the low half
-    auto place_by_id = [&](int id, unsigned key, int slot) {
+    auto place_by_id = [&](int id, unsigned key, int slot, int ord) {
       const int q = id >> 16, j1 = id & 0xffff;
       if (j1 == 0) place_stay(q, key, slot);
-      else place_ext(q, ext_token(j1 - 1), key, slot);
+      else place_ext(q, ext_token(j1 - 1), key, slot, ord);
     };
 
     // the cut as scores (bin edges): score > f_hi is above the cut bin, score > f_lo is in it
@@ -911,8 +924,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           list_id[li] = id;
         }
       };
-      if (is_stay && NS <= kOwnStayLanes && !kWide) {
-        // At most four stay warps: each looks at all (at most 128) stay candidates itself, so
+      if (is_stay && K <= NS && NS <= kOwnStayLanes && !kWide) {
+        // Every beam entry has a stay lane of its own, in at most four stay warps: each looks at all (at most 128) stay candidates itself, so
         // the places follow from ballots alone and no counter is shared.
         int before = 0, total_sel = 0;  // selected stays in the warps below this one / in all
         float sc = neg_inf();
@@ -1010,7 +1023,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       // ranks the members of the cut bin exactly (score, then candidate id) and writes the
       // winners to the slots between the stays and the extensions.
       const int n_stay = min(sc_c[SC_SLOT], K);
-      if (is_stay && NS <= kOwnStayLanes && !kWide) {
+      if (is_stay && K <= NS && NS <= kOwnStayLanes && !kWide) {
         const int slot = __float_as_int(kc[1]);
         if (slot >= 0) place_stay(tid, score_key(kc[0]), slot);
       } else if (is_stay) {
@@ -1019,19 +1032,31 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         const int n_ext = min(sc_c[SC_SLOT_E], K);
         for (int x = xl; x < n_ext; x += NX) {
           const int slot = nbn - 1 - x;
-          if (slot >= 0) place_by_id(sel_id[slot], sel_key[slot], slot);
+          if (slot >= 0) place_by_id(sel_id[slot], sel_key[slot], slot, x);
         }
       } else {
-        for (int li = lane; li < n_listed; li += 32) {
-          const unsigned key = list_key[li];
-          const int id = list_id[li];
-          int rank = 0;
-          for (int j = 0; j < n_listed; ++j) {
-            const unsigned kj = list_key[j];
-            rank += (kj > key || (kj == key && list_id[j] < id)) ? 1 : 0;
+        // (the extensions among the winners are numbered after those placed above)
+        const int n_ext = min(sc_c[SC_SLOT_E], K);
+        int won_ext = 0;
+        for (int base = 0; base < n_listed; base += 32) {
+          const int li = base + lane;
+          unsigned key = 0u;
+          int id = 0, rank = 0x7fffffff;
+          if (li < n_listed) {
+            key = list_key[li];
+            id = list_id[li];
+            rank = 0;
+            for (int j = 0; j < n_listed; ++j) {
+              const unsigned kj = list_key[j];
+              rank += (kj > key || (kj == key && list_id[j] < id)) ? 1 : 0;
+            }
           }
-          if (rank < n_winners) place_by_id(id, key, n_stay + rank);
+          const bool won = rank < n_winners;
+          const unsigned mx = __ballot_sync(kFull, won && (id & 0xffff) != 0);
+          if (won) place_by_id(id, key, n_stay + rank, n_ext + won_ext + __popc(mx & lt_mask));
+          won_ext += __popc(mx);
         }
+        if (lane == 0) scal[SC_MADE + par] = n_ext + won_ext;  // new prefixes of this frame
       }
     } else {
       // ---- exact fallback: radix select over the integer keys ------------------------
@@ -1093,18 +1118,22 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           if (r_all || eq_rank < need) slot = total_gt + eq_rank;
           ++eq_rank;
         }
-        if (slot >= 0) place_by_id(id, key, slot);
+        if (slot >= 0)
+          place_by_id(id, key, slot, (id & 0xffff) ? atomicAdd(&sc_c[SC_SLOT_E], 1) : 0);
       });
+      __syncthreads();
+      if (tid == 0) scal[SC_MADE + par] = sc_c[SC_SLOT_E];
     }
     if (cut.total == 0) status |= 8;  // FLTOP_ST_EMPTY_BEAM
     offset += (double)best;
     __syncthreads();  // B4: the next beam and its hash table are complete
 
     // (chore warp) what the next frame has to write out
+    const int made = min(scal[SC_MADE + par], K);  // new prefixes: consecutive node ids
     pend_at = n_nodes;
-    pend_bytes = (arena_ok && nbn > 0) ? (unsigned)(((nbn + 1) & ~1) * sizeof(TrieNode)) : 0u;
-    if (!arena_ok && nbn > 0) status |= 2;  // FLTOP_ST_ARENA_FULL
-    n_nodes += (nbn + 1) & ~1;
+    pend_bytes = (arena_ok && made > 0) ? (unsigned)(((made + 1) & ~1) * sizeof(TrieNode)) : 0u;
+    if (!arena_ok && made > 0) status |= 2;  // FLTOP_ST_ARENA_FULL
+    if (arena_ok) n_nodes += (made + 1) & ~1;
     live_sum += nbn;
     nb = nbn;
     cur = nxt;
@@ -1128,10 +1157,12 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   status |= scal[SC_STATUS];
   if (p.stats) {
     if (created) atomicAdd(&scal[SC_CREATED], created);
+    if (tag_clashes) atomicAdd(&scal[SC_CLASHES], tag_clashes);
     __syncthreads();
     if (tid == 0) {
-      int32_t* o = p.stats + 4 * (int64_t)b;
+      int32_t* o = p.stats + kStatWords * (int64_t)b;
       o[0] = len; o[1] = scal[SC_CREATED]; o[2] = live_sum - scal[SC_DEAD]; o[3] = n_nodes;
+      o[4] = scal[SC_CLASHES]; o[5] = 0;
     }
   }
 
@@ -1157,6 +1188,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       hd->nbeam = nb; hd->n_nodes = n_nodes; hd->frames = frames_seen;
       hd->status = status & ~1;  // a bad chunk length is not sticky
       hd->offset = offset;
+      hd->drift = 0;
     }
   }
 

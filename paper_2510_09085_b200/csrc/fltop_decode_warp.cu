@@ -131,7 +131,12 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       const unsigned long long h = e_print;
       const unsigned val = (((unsigned)h & 0xfffffu) << 12) | (unsigned)lane;
       unsigned pos = (unsigned)(h >> 40) & (kWarpTab - 1);
-      while (atomicCAS(&S.tab[pos], kFree, val) != kFree) pos = (pos + 1) & (kWarpTab - 1);
+      bool in = false;
+      for (int probes = 0; probes < kWarpTab && !in; ++probes) {
+        in = atomicCAS(&S.tab[pos], kFree, val) == kFree;
+        pos = (pos + 1) & (kWarpTab - 1);
+      }
+      if (!in) status |= 16;  // FLTOP_ST_INTERNAL (cannot happen: 32 entries, 128 slots)
     }
   };
   auto table_find = [&](const BeamCopy& c, unsigned long long h) -> int {
@@ -189,6 +194,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       kept = chosen;
     }
     kept_sum += __popc(kept);
+    if (p.dbg_masks && lane == 0) p.dbg_masks[(int64_t)b * p.T + t] = kept;  // instrumented launches only
     const bool blank_kept = (kept >> blank) & 1u;
     const float lp_blank_raw = __shfl_sync(kFull, lp, blank);
     const float lp_blank = blank_kept ? lp_blank_raw : neg_inf();
@@ -235,13 +241,15 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
     const float best = -(float)(cut.first * kBinsPerLane) * (1.f / kBinsPerNat);
     const bool take_all = cut.cut_count == cut.left;  // also when there is no cut at all
     const int nbn = min(cut.total, K);
+    int n_new = 0;  // new prefixes of this frame so far
     const bool arena_ok = (int64_t)n_nodes + ((K + 1) & ~1) <= p.nodes_per_utt;
     const unsigned my_dup = S.dupw[lane];
 
-    // Writing a candidate into slot `slot` of the next beam: q = 0 stays as it is, q > 0
-    // (token + 1) is a new prefix and gets its trie record.
-    auto place = [&](int q, int c_plus1, float sc, int slot) {
-      if ((unsigned)slot >= (unsigned)K) return;  // only reachable with NaN scores
+    // Writing a candidate into slot `slot` of the next beam: c_plus1 = 0 stays as it is,
+    // c_plus1 > 0 (token + 1) is a new prefix and gets its trie record; `ord` numbers the new
+    // prefixes of the frame, which get consecutive node ids.
+    auto place = [&](int q, int c_plus1, float sc, int slot, int ord) {
+      if ((unsigned)slot >= (unsigned)K || (unsigned)ord >= (unsigned)K) return;  // (NaN scores)
       if (c_plus1 == 0) {
         N.last[slot] = C.last[q];
         N.pb[slot] = S.st_pb[q] - best;
@@ -260,9 +268,9 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
         N.tot[slot] = sc - best;
         N.print[slot] = child_print(pp, c);
         N.pprint[slot] = pp;
-        N.node[slot] = arena_ok ? n_nodes + slot : 0;  // arena full: nothing to walk back to
+        N.node[slot] = arena_ok ? n_nodes + ord : 0;  // arena full: nothing to walk back to
         N.len[slot] = C.len[q] + 1;
-        if (arena_ok) nodes[n_nodes + slot] = TrieNode{C.node[q], c};
+        if (arena_ok) nodes[n_nodes + ord] = TrieNode{C.node[q], c};
         ++created;
       }
     };
@@ -279,17 +287,17 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       N.node[slot] = e_node;
       N.len[slot] = e_len;
     };
-    auto place_own_ext = [&](int c, float sc, int slot) {
-      if ((unsigned)slot >= (unsigned)K) return;
+    auto place_own_ext = [&](int c, float sc, int slot, int ord) {
+      if ((unsigned)slot >= (unsigned)K || (unsigned)ord >= (unsigned)K) return;
       N.last[slot] = c;
       N.pb[slot] = neg_inf();
       N.pnb[slot] = sc - best;
       N.tot[slot] = sc - best;
       N.print[slot] = child_print(e_print, c);
       N.pprint[slot] = e_print;
-      N.node[slot] = arena_ok ? n_nodes + slot : 0;
+      N.node[slot] = arena_ok ? n_nodes + ord : 0;
       N.len[slot] = e_len + 1;
-      if (arena_ok) nodes[n_nodes + slot] = TrieNode{e_node, c};
+      if (arena_ok) nodes[n_nodes + ord] = TrieNode{e_node, c};
       ++created;
     };
 
@@ -322,7 +330,10 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
         if ((my_dup >> c) & 1u) sc = neg_inf();  // merged into a stay candidate
         const bool x_sure = sc > f_hi, x_list = !x_sure && sc > f_lo;
         const unsigned bx = __ballot_sync(kFull, x_sure);
-        if (x_sure) place_own_ext(c, sc, nbn - 1 - (n_ext + __popc(bx & lt_mask)));
+        if (x_sure) {
+          const int ord = n_ext + __popc(bx & lt_mask);
+          place_own_ext(c, sc, nbn - 1 - ord, ord);
+        }
         n_ext += __popc(bx);
         const unsigned bl = __ballot_sync(kFull, x_list);
         if (x_list) {
@@ -336,17 +347,28 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       }
       __syncwarp();
       // the members of the cut bin, ranked by (score, candidate id): the best `left` go in between
+      n_new = n_ext;
       if (!take_all) {
         const int n = min(n_list, kListCap);
-        for (int li = lane; li < n; li += 32) {
-          const unsigned key = S.list_key[li];
-          const int id = S.list_id[li];
-          int rank = 0;
-          for (int j = 0; j < n; ++j) {
-            const unsigned kj = S.list_key[j];
-            rank += (kj > key || (kj == key && S.list_id[j] < id)) ? 1 : 0;
+        for (int base = 0; base < n; base += 32) {
+          const int li = base + lane;
+          unsigned key = 0u;
+          int id = 0, rank = 0x7fffffff;
+          if (li < n) {
+            key = S.list_key[li];
+            id = S.list_id[li];
+            rank = 0;
+            for (int j = 0; j < n; ++j) {
+              const unsigned kj = S.list_key[j];
+              rank += (kj > key || (kj == key && S.list_id[j] < id)) ? 1 : 0;
+            }
           }
-          if (rank < cut.left) place(id >> 16, id & 0xffff, key_score(key), n_stay + rank);
+          const bool won = rank < cut.left;
+          const unsigned mx = __ballot_sync(kFull, won && (id & 0xffff) != 0);
+          if (won)
+            place(id >> 16, id & 0xffff, key_score(key), n_stay + rank,
+                  n_new + __popc(mx & lt_mask));
+          n_new += __popc(mx);
         }
       }
     } else {
@@ -393,16 +415,20 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
         const unsigned key = score_key(sc);
         const bool above = key > kth, tie = key == kth && kth != 0u;
         const unsigned ba = __ballot_sync(kFull, above);
-        if (above) place_own_ext(c, sc, nbn - 1 - (n_ext + __popc(ba & lt_mask)));
+        if (above) place_own_ext(c, sc, nbn - 1 - (n_ext + __popc(ba & lt_mask)),
+                                 n_new + __popc(ba & lt_mask));
         n_ext += __popc(ba);
+        n_new += __popc(ba);
         const unsigned bt = __ballot_sync(kFull, tie);
         const int r = n_tie + __popc(bt & lt_mask);
-        if (tie && r < need) place_own_ext(c, sc, n_above_stay + r);
+        const unsigned taken = __ballot_sync(kFull, tie && r < need);
+        if (tie && r < need) place_own_ext(c, sc, n_above_stay + r, n_new + __popc(taken & lt_mask));
+        n_new += __popc(taken);
         n_tie = min(n_tie + __popc(bt), need);
       }
     }
     if (cut.total == 0) status |= 8;  // FLTOP_ST_EMPTY_BEAM
-    if (!arena_ok && nbn > 0) status |= 2;  // FLTOP_ST_ARENA_FULL
+    if (!arena_ok && n_new > 0) status |= 2;  // FLTOP_ST_ARENA_FULL
     __syncwarp();
 
     // ---- the next beam becomes the beam -----------------------------------------------------
@@ -414,7 +440,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       e_print = N.print[lane]; e_pprint = N.pprint[lane]; e_node = N.node[lane]; e_len = N.len[lane];
     }
     offset += (double)best;
-    n_nodes += (nbn + 1) & ~1;
+    if (arena_ok) n_nodes += (n_new + 1) & ~1;
     live_sum += nbn;
     nb = nbn;
     cur ^= 1;
@@ -423,6 +449,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
     __syncwarp();
   }
   frames_seen += len;
+  status = (int)__reduce_or_sync(kFull, (unsigned)status);  // a lane's flag is the warp's
 
   // survivor counts per frame are not kept: the utterance's total stands in the first place
   {
@@ -432,8 +459,8 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
   if (p.stats) {
     const int made = __reduce_add_sync(kFull, created);
     if (lane == 0) {
-      int32_t* o = p.stats + 4 * (int64_t)b;
-      o[0] = len; o[1] = made; o[2] = live_sum; o[3] = n_nodes;
+      int32_t* o = p.stats + kStatWords * (int64_t)b;
+      o[0] = len; o[1] = made; o[2] = live_sum; o[3] = n_nodes; o[4] = 0; o[5] = 0;
     }
   }
 
@@ -452,6 +479,7 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
       hd->nbeam = nb; hd->n_nodes = n_nodes; hd->frames = frames_seen;
       hd->status = status & ~1;  // a bad chunk length is not sticky
       hd->offset = offset;
+      hd->drift = 0;
     }
   }
 

@@ -26,7 +26,9 @@ struct StateHeader {
   int32_t frames;     // frames consumed since the last reset
   int32_t status;     // sticky FLTOP_ST_* bits
   double offset;      // log-probability of the renormalisation point (see decode kernel)
-  int32_t pad[2];
+  int32_t drift;      // float bits: how far blank-only frames have let the relative scores sink
+                      // since the point was last moved (row kernel; 0 from the others)
+  int32_t pad;
 };
 constexpr int kStateHeaderWords = sizeof(StateHeader) / 4;
 // beam arrays stored after the header, each K words (fingerprints: 2K words each):
@@ -81,8 +83,17 @@ struct DecodeParams {
   float* out_scores;        // [B,K]
   int32_t* out_nhyp;        // [B]
   int32_t* out_status;      // [B] or null
-  int32_t* stats;           // [B,4] frames, trie nodes created, sum of beam sizes, node ids used; or null
+  int32_t* stats;           // [B,kStatWords] (see below) or null
+  int32_t table_slots;      // 0, or a power of two: the fingerprint table is cut down to this many
+                            // slots (the test of the bounded probe walks makes it overflow)
+  // instrumented instantiations (tests and profiling; null in every ordinary launch)
+  uint32_t* dbg_masks;      // [B*T] survivor mask of every frame a decode kernel pruned itself
+  long long* dbg_clocks;    // [dbg_frames][32 warps][8 phases] clock64 of block 0
+  int32_t dbg_frame0, dbg_frames;
 };
+// per-utterance statistics of a call: frames, trie nodes created, sum of beam sizes, node ids
+// used, fingerprint-tag clashes (probes that met another sequence with the same 20-bit tag)
+constexpr int kStatWords = 8;
 
 size_t decode_smem_bytes(int K, int V);
 int decode_block_threads(int K, int V, bool pruning, int top_n, bool latency_bound);
@@ -90,6 +101,9 @@ cudaError_t launch_prune(const PruneParams& p, cudaStream_t s);
 // keeps at most top_n survivors per frame (no-op for top_n <= 0 or >= V)
 cudaError_t launch_topn_cap(const PruneParams& p, int top_n, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s);
+// character vocabularies, beams up to 64, rows pruned inside (fltop_decode_rows.cu)
+bool decode_rows_eligible(const DecodeParams& p);
+cudaError_t launch_decode_rows(const DecodeParams& p, cudaStream_t s);
 // narrow beams over narrow vocabularies: one warp per utterance (fltop_decode_warp.cu)
 bool decode_warp_eligible(const DecodeParams& p);
 cudaError_t launch_decode_warp(const DecodeParams& p, cudaStream_t s);

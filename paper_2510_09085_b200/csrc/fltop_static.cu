@@ -91,7 +91,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   pp.counts = reinterpret_cast<int32_t*>(scratch);
   pp.entries = reinterpret_cast<Survivor*>(scratch + kCountsBytes);
 
-  DecodeParams dp;
+  DecodeParams dp = {};
   dp.lengths = d_lengths; dp.flags = nullptr; dp.B = B; dp.T = T; dp.V = vocab_size;
   dp.K = beam_width; dp.blank = blank_id; dp.L = max_out_len; dp.streaming = 0;
   dp.emit_default = 1; dp.block_threads = 0; dp.co_resident = 0; dp.warp_mode = 0; dp.pruning = threshold_r >= 5e-4f ? 1 : 0;

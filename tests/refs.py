@@ -128,3 +128,42 @@ def py_decode(lp: np.ndarray, blank: int, K: int, log_r: np.float32 | None, top_
             surv = sorted(c for c in cand if lp[t, c] >= thr)
         s.step(lp[t], surv)
     return s
+
+
+def ctc_forward_logprob(lp: np.ndarray, seq, blank: int, keep: np.ndarray | None = None) -> float:
+    """log P(seq | lp) by the textbook CTC forward (alpha) recursion in float64.
+
+    ``lp`` [T,V] log-probabilities; ``keep`` [T,V] (bool) restricts every frame to its surviving
+    tokens (the others get probability 0).  This is the sum over ALL alignments of ``seq``, so it
+    is an upper bound of what any beam search can assign to ``seq`` on the same frames."""
+    lp = np.asarray(lp, dtype=np.float64)
+    if keep is not None:
+        lp = np.where(keep, lp, -np.inf)
+    T = lp.shape[0]
+    ext = [blank]
+    for c in seq:
+        ext += [int(c), blank]
+    ext = np.asarray(ext, dtype=np.int64)
+    S = len(ext)
+    # a state may be entered from two states back iff it is a label that differs from the
+    # label two states back (blanks and repeated labels may not be skipped over)
+    skip = np.zeros(S, dtype=bool)
+    skip[2:] = (ext[2:] != blank) & (ext[2:] != ext[:-2])
+    alpha = np.full(S, -np.inf)
+    if T == 0:
+        return 0.0 if S == 1 else -np.inf
+    if S == 1:  # the empty labelling: blank at every frame
+        return float(lp[:, blank].sum())
+    alpha[0] = lp[0, blank]
+    if S > 1:
+        alpha[1] = lp[0, ext[1]]
+    with np.errstate(invalid="ignore", divide="ignore"):
+        for t in range(1, T):
+            a1 = np.concatenate(([-np.inf], alpha[:-1]))
+            a2 = np.where(skip, np.concatenate(([-np.inf, -np.inf], alpha[:-2])), -np.inf)
+            m = np.maximum(alpha, np.maximum(a1, a2))
+            tot = np.where(np.isfinite(m),
+                           m + np.log(np.exp(alpha - m) + np.exp(a1 - m) + np.exp(a2 - m)), -np.inf)
+            alpha = tot + lp[t, ext]
+        last = np.logaddexp(alpha[-1], alpha[-2])
+    return float(last)

@@ -74,7 +74,7 @@ def test_decode_of_half_precision_rows_matches_oracle(dtype, V, K, r, kw):
     T = em.shape[1]
     ln[:] = [0, 1, T, 37, 64]
     x, wide = _narrow(em, dtype)
-    res = oracle.decode(wide, ln, 0, K, r, **kw)
+    res = oracle.decode(wide, ln, 0, K, r, want_masks=True, **kw)
     outs = []
     for fusion in (1, 0):
         d = _binding().Decoder(V, 0, K, r, B, max(T, 1), emission_dtype=dtype, **kw)
@@ -91,12 +91,13 @@ def test_decode_of_half_precision_rows_matches_oracle(dtype, V, K, r, kw):
         loose = 0.5 if (dtype == torch.bfloat16 and kw.get("merge_max")) else 0.0
         for b in range(B):
             check_hyps(d.hyps(b), res.hyps(b), K, max_unmatched_frac=loose,
-                       where=f"{dtype} V={V} fusion={fusion} utt {b}")
+                       where=f"{dtype} V={V} fusion={fusion} utt {b}", lp=wide[b, : ln[b]],
+                       keep=res.keep[b, : ln[b]], cascade=0.5)
         outs.append(d)
     # (coarse bf16 values tie often: which of two equal-scoring hypotheses comes first, or
     # makes the cut, is not unique - the scores are)
     if not kw.get("merge_max"):
-        assert torch.equal(outs[0].scores[:B], outs[1].scores[:B])
+        assert torch.allclose(outs[0].scores[:B], outs[1].scores[:B], rtol=0, atol=1e-4)
     for d in outs:
         d.close()
 

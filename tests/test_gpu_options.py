@@ -41,12 +41,14 @@ def _compare(em, ln, K, r, top_n=0, theta=0.0, frac=0.0, merge_max=False):
     torch.cuda.synchronize()
     assert (d.status.cpu().numpy()[:B] == 0).all()
     st = d.last_call_stats()
-    res = oracle.decode(em, ln, 0, K, r, top_n=top_n, beam_threshold=theta, merge_max=merge_max)
+    res = oracle.decode(em, ln, 0, K, r, top_n=top_n, beam_threshold=theta, merge_max=merge_max,
+                        want_masks=True)
     res.mean_live = st["live_hypotheses_sum"] / max(1, st["frames"])
     for b in range(B):
         g, o = d.hyps(b), res.hyps(b)
         if theta <= 0:
-            check_hyps(g, o, K, max_unmatched_frac=frac, where=f"utt {b}")
+            check_hyps(g, o, K, max_unmatched_frac=frac, where=f"utt {b}", lp=em[b, : ln[b]],
+                       keep=res.keep[b, : ln[b]])
             continue
         gm, om = dict(g), dict(o)
         assert g[0][0] == o[0][0] or abs(o[0][1] - o[1][1]) < TOL

@@ -32,11 +32,13 @@ def compare_batch(em, ln, blank, K, r, utterances=None, max_unmatched_frac=0.0):
     status = d.status.cpu().numpy()
     sel = range(len(ln)) if utterances is None else utterances
     assert (status[: len(ln)] == 0).all(), status
-    res = oracle.decode(em[list(sel)], np.asarray(ln)[list(sel)], blank, K, r)
+    res = oracle.decode(em[list(sel)], np.asarray(ln)[list(sel)], blank, K, r, want_masks=True)
     swaps = 0
     for i, b in enumerate(sel):
+        n = int(ln[b])
         swaps += check_hyps(d.hyps(b), res.hyps(i), K, max_unmatched_frac=max_unmatched_frac,
-                            where=f"utt {b} K={K} r={r}")
+                            where=f"utt {b} K={K} r={r}", lp=em[b, :n], keep=res.keep[i, :n],
+                            blank=blank)
     d.close()
     return swaps
 
@@ -218,10 +220,10 @@ def test_many_near_equal_scores_take_the_exact_select_path():
     ln = np.array([T, T - 3, 5], dtype=np.int32)
     for K, r in [(8, 0.0), (20, 0.5), (100, 0.0)]:
         d = gpu_decode(em, ln, 0, K, r)
-        res = oracle.decode(em, ln, 0, K, r)
+        res = oracle.decode(em, ln, 0, K, r, want_masks=True)
         for b in range(B):
             check_hyps(d.hyps(b), res.hyps(b), K, max_unmatched_frac=0.3,
-                       where=f"flat utt {b} K={K}")
+                       where=f"flat utt {b} K={K}", lp=em[b, : ln[b]], keep=res.keep[b, : ln[b]])
         d.close()
 
 
@@ -240,7 +242,7 @@ def test_wide_beam_with_a_crowded_cut_bin(spread):
         res = oracle.decode(em, ln, 0, K, 0.0)
         for b in range(B):
             check_hyps(d.hyps(b), res.hyps(b), K, max_unmatched_frac=0.3,
-                       where=f"flat wide utt {b} K={K} spread={spread}")
+                       where=f"flat wide utt {b} K={K} spread={spread}", lp=em[b, : ln[b]])
         d.close()
 
 

@@ -111,6 +111,7 @@ def test_serving_workload_sampled():
     torch.cuda.synchronize()
     assert (d.status.cpu().numpy() == 0).all()
     sample = [0, 1, 511, 1023]
-    res = oracle.decode(wl.emissions[sample], wl.lengths[sample], 0, K, r)
+    res = oracle.decode(wl.emissions[sample], wl.lengths[sample], 0, K, r, want_masks=True)
     for i, s in enumerate(sample):
-        check_hyps(d.hyps(s), res.hyps(i), K, max_unmatched_frac=0.25, where=f"stream {s}")
+        check_hyps(d.hyps(s), res.hyps(i), K, max_unmatched_frac=0.25, where=f"stream {s}",
+                   lp=wl.emissions[s], keep=res.keep[i])
