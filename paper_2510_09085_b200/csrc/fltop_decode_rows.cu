@@ -98,7 +98,7 @@ struct __align__(16) CutOut {
   int n_listed;    // members of the cut bin if it has to be split, else 0
   int left;        // how many of them are kept
   int empty;       // 1: no candidate at all
-  int pad;
+  int thr;         // the cut bin
 };
 
 // One warp turns the score histogram into the cut (all lanes get the result).  Lane l owns bins
@@ -203,6 +203,8 @@ struct RowsSmem {
   unsigned dupw[2][KMAX];                   // bit c of word q: "entry q extended by c" is merged
   unsigned tab[2][kTable];
   unsigned hist[kFastBins];
+  unsigned hist2[kFastBins];                // the members of a crowded cut bin, binned once more
+  int cut2[4];                              // ... and what the scan of that found
   unsigned list_key[kListCap];
   int list_id[kListCap];
   float list_pb[kListCap], list_pnb[kListCap];  // of listed stay candidates
@@ -287,7 +289,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   // ---- initialise shared state ---------------------------------------------------------
   for (int i = tid; i < 2 * KMAX; i += NT) (&S.dupw[0][0])[i] = 0u;
   for (int i = tid; i < 2 * kTable; i += NT) (&S.tab[0][0])[i] = kNoEntry;
-  for (int i = tid; i < kFastBins; i += NT) S.hist[i] = 0u;
+  for (int i = tid; i < kFastBins; i += NT) { S.hist[i] = 0u; S.hist2[i] = 0u; }
   if (tid < 2 * FS_COUNT) (&S.fs[0][0])[tid] = 0;
   if (tid < BS_COUNT) S.bs[tid] = 0;
   int cur = 0, nb, n_nodes, frames_seen;
@@ -435,9 +437,10 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   int round = 0;  // block-wide counts taken by the exact fallback so far (its counters rotate)
   int g = 0;      // frames that went through selection so far (its buffers alternate)
   float drift = drift0;  // how far blank-only frames have let the scores sink since
+  FrameHead head_next = S.head[0];
   for (int t = 0; t < len; ++t) {
-    // the frame as the chore warp prepared it
-    const FrameHead head = S.head[t & 3];
+    // the frame as the chore warp prepared it (read before the last barrier of frame t-1)
+    const FrameHead head = head_next;
     // Chore warp, while the others evaluate: the trie records of the last selection leave,
     // the row of frame t+3 is requested.
     auto chore_window = [&]() {
@@ -468,6 +471,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
       drift += head.lp_blank;
       pend_bytes = 0u;
       live_sum += nb;
+      head_next = S.head[(t + 1) & 3];  // prepared a frame ago
       __syncthreads();
       continue;
     }
@@ -492,6 +496,8 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     const int n_trows = (head.snb + (1 << lgT) - 1) >> lgT;  // token rows of this frame
     // position (among the surviving non-blank tokens) of the token of this lane's k-th row
     auto row_token = [&](int k) -> int { return ((part + k * P) << lgT) + jsub; };
+    // (with few survivors most extension warps have no row at all and sit the frame out)
+    const bool has_rows = is_ext && part < n_trows;
 
     // ---- P1: every candidate is evaluated once and counted ---------------------------------
     // Extension lanes keep the scores of their first rows in registers, and what their best
@@ -512,6 +518,9 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     Where swh = Where{0, 0};
     float npb = neg_inf(), npnb = neg_inf(), stot = neg_inf();
     float s_own = neg_inf(), s_dup = neg_inf();
+    float other_tot[KMAX / 32];  // the stay candidates of lane `lane` of every stay warp
+#pragma unroll
+    for (int w = 0; w < KMAX / 32; ++w) other_tot[w] = neg_inf();
     if (is_stay) {
       if (tid < nb) {
         se = hc[tid];
@@ -537,7 +546,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         s_dup = dup;
       }
       if (tid < KMAX) S.st_tot[tid] = stot;
-    } else if (is_ext) {
+    } else if (has_rows) {
       if (xq < nb) {
         se = hc[xq];
         hp = id_c[xq].print;
@@ -588,30 +597,94 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         o.n_listed = all ? 0 : c.cut_count;
         o.left = c.left;
         o.empty = c.total == 0 ? 1 : 0;
-        o.pad = 0;
+        o.thr = c.thr;
         S.cut = o;
       }
     } else {
-      const uint4 ones = make_uint4(~0u, ~0u, ~0u, ~0u);
-      uint4* const t_n = reinterpret_cast<uint4*>(tab_n);
-      for (int i = tid; i < kTable / 4; i += NT - 32) t_n[i] = ones;
-      if (is_stay && tid < nb) {
-        // what a stay candidate needs only if it is kept: worked out while the scan runs
-        npnb = lse2(s_own, s_dup);
-        swh = wh_c[tid];
+      if (is_stay) {
+        const uint4 ones = make_uint4(~0u, ~0u, ~0u, ~0u);
+        uint4* const t_n = reinterpret_cast<uint4*>(tab_n);
+        for (int i = tid; i < kTable / 4; i += 32 * nsw) t_n[i] = ones;
+        // what a stay candidate needs only if it is kept, and the other stay warps'
+        // candidates: fetched and worked out while the scan runs
+        if (tid < nb) {
+          npnb = lse2(s_own, s_dup);
+          swh = wh_c[tid];
+        }
+#pragma unroll
+        for (int w = 0; w < KMAX / 32; ++w) other_tot[w] = (w < nsw) ? S.st_tot[w * 32 + lane] : neg_inf();
+      } else if (is_ext && sc1 != neg_inf()) {
+        // an extension that a stay candidate has absorbed (the merge) is no candidate
+        if ((dupw[xq] >> tok1) & 1u) sc1 = neg_inf();
       }
     }
     clock_mark(t, 3);
     __syncthreads();  // B2: the cut is known
     const CutOut cut = S.cut;
     const float best = cut.best, f_lo = cut.f_lo, f_hi = cut.f_hi;
-    const int n_listed = cut.n_listed, nbn = cut.nbn;
+    int n_listed = cut.n_listed, left = cut.left;
+    const int nbn = cut.nbn;
     const bool arena_ok = n_nodes + ((K + 1) & ~1) <= nodes_cap;
+
+    // A crowded cut bin (more members than the pairwise ranking takes) is binned once more:
+    // an inner bin into 256 sub-bins over its quarter nat, the last bin - everything more
+    // than 63.75 nats below the reference, where the hopeless candidates of a sharply peaked
+    // utterance collect - into quarter-nat bins over the next 64 nats.  The cut is then
+    // located among those and only that sub-bin's members are ranked.
+    const bool refined = n_listed > kListCap;  // block-uniform
+    const float hi_edge = -(float)cut.thr * (1.f / kBinsPerNat);
+    const float sub_scale = cut.thr >= kFastBins - 1 ? kBinsPerNat : kBinsPerNat * (float)kFastBins;
+    int sub_thr = 0;
+    bool sub_all = false;
+    auto sub_bin = [&](float sc) -> int {
+      const int b2 = __float2int_rz((hi_edge - sc) * sub_scale);
+      return min(kFastBins - 1, max(0, b2));
+    };
+    // 2: the candidate is kept, 1: it is in the (sub-)bin that the cut runs through, 0: it is out
+    auto klass = [&](float sc) -> int {
+      if (sc > f_hi) return 2;
+      if (!(sc > f_lo)) return 0;
+      if (!refined) return 1;
+      const int sb = sub_bin(sc);
+      return sb < sub_thr ? 2 : (sb == sub_thr ? (sub_all ? 2 : 1) : 0);
+    };
+    if (refined) {
+      auto count2 = [&](float sc) {
+        if (sc > f_lo && !(sc > f_hi)) atomicAdd(&S.hist2[sub_bin(sc)], 1u);
+      };
+      if (is_stay) {
+        count2(stot);
+      } else if (is_ext && xq < nb) {
+        const unsigned dw = dupw[xq];
+        for (int k = 0; part + k * P < n_trows; ++k) {
+          const TokLp tl = tokj[row_token(k)];
+          if (tl.tok >= 0 && !((dw >> tl.tok) & 1u))
+            count2(((tl.tok == se.last) ? se.pb : se.tot) + tl.lp);
+        }
+      }
+      __syncthreads();
+      if (is_chore) {
+        const Cut c2 = scan_score_histogram_ballots<7>(S.hist2, left);
+        if (lane == 0) {
+          S.cut2[0] = c2.thr; S.cut2[1] = c2.left; S.cut2[2] = c2.cut_count;
+          S.cut2[3] = c2.cut_count == c2.left ? 1 : 0;
+        }
+        __syncwarp();
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        reinterpret_cast<uint4*>(S.hist2)[lane] = zero;
+        reinterpret_cast<uint4*>(S.hist2)[lane + 32] = zero;
+      }
+      __syncthreads();
+      sub_thr = S.cut2[0];
+      sub_all = S.cut2[3] != 0;
+      left = S.cut2[1];
+      n_listed = sub_all ? 0 : S.cut2[2];
+    }
     if ((HOOKS & 2) && b == 0 && tid == 0 && p.dbg_clocks && t >= p.dbg_frame0 &&
         t < p.dbg_frame0 + p.dbg_frames) {
       // (rows 24.. of the record are free: fewer than 24 warps) what the scan found
       long long* const o = p.dbg_clocks + ((int64_t)(t - p.dbg_frame0) * 32 + 24) * 8;
-      o[0] = nbn; o[1] = n_listed; o[2] = cut.left; o[3] = cut.empty; o[4] = nb;
+      o[0] = nbn; o[1] = n_listed; o[2] = left; o[3] = cut.empty; o[4] = nb;
       o[5] = head.snb; o[6] = n_trows; o[7] = 0;
     }
 
@@ -680,8 +753,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
 #pragma unroll
         for (int w = 0; w < KMAX / 32; ++w) {
           if (w < nsw) {
-            const float s_w = (w == warp) ? stot : S.st_tot[w * 32 + lane];
-            const int k_w = s_w > f_hi ? 2 : (s_w > f_lo ? 1 : 0);
+            const int k_w = klass(other_tot[w]);
             const unsigned m_w = __ballot_sync(kFull, k_w == 2);
             const int n_w = __popc(m_w);
             before += w < warp ? n_w : 0;
@@ -709,12 +781,12 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
             S.list_pnb[at] = npnb;
           }
         }
-      } else if (is_ext) {
+      } else if (has_rows) {
         // this lane's best candidate first (its token and fingerprint are ready) ...
-        bool in1 = sc1 > f_lo;
-        if (__any_sync(kFull, in1)) {
-          if (in1) in1 = !((dupw[xq] >> tok1) & 1u);  // not merged into a stay candidate
-          const bool sure1 = in1 && sc1 > f_hi;
+        const int kl1 = klass(sc1);
+        const bool in1 = kl1 != 0;
+        if (__any_sync(kFull, in1 || sc2 > f_lo)) {
+          const bool sure1 = kl1 == 2;
           const int ord = take_places(sure1, &fs[FS_SLOT_E]);
           if (sure1) place_new(hp, xwh, tok1, h1, sc1, nbn - 1 - ord, ord);
           if (n_listed > 0) {
@@ -729,8 +801,9 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
 #pragma unroll
               for (int k = 0; k < kRowCache; ++k) {
                 if (kc[k] > f_lo && row_token(k) != j1 && !((dw >> tokj[row_token(k)].tok) & 1u)) {
-                  if (kc[k] > f_hi) sure |= 1u << k;
-                  else lst |= 1u << k;
+                  const int kl = klass(kc[k]);
+                  if (kl == 2) sure |= 1u << k;
+                  else if (kl == 1) lst |= 1u << k;
                 }
               }
             }
@@ -765,7 +838,8 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
           const int tok = tl.tok;
           float sc = ((tok == se.last) ? se.pb : se.tot) + tl.lp;
           if (sc > f_lo && ((dupw[xq] >> tok) & 1u)) sc = neg_inf();
-          const bool isin = sc > f_lo, issure = sc > f_hi;
+          const int kl = klass(sc);
+          const bool isin = kl != 0, issure = kl == 2;
           if (__any_sync(kFull, isin)) {
             const int ord = take_places(issure, &fs[FS_SLOT_E]);
             if (issure) place_ext(xq, tok, sc, nbn - 1 - ord, ord);
@@ -801,7 +875,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
           if (n > 32)
             rank += __popc(__ballot_sync(
                 kFull, lane + 32 < n && (key_b > key || (key_b == key && id_b < id))));
-          if (rank < cut.left) {
+          if (rank < left) {
             if (lane == n_won) { my_m = m; my_rank = rank; }
             ++n_won;
           }
@@ -887,6 +961,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     if (cut.empty) status |= 8;  // FLTOP_ST_EMPTY_BEAM
     if (is_stay) offset += (double)best;  // (the stay lanes write the scores out)
     clock_mark(t, 6);
+    head_next = S.head[(t + 1) & 3];  // prepared a frame ago
     __syncthreads();  // B4: the next beam and its table are complete
     clock_mark(t, 7);
 

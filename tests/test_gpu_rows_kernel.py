@@ -8,6 +8,7 @@ import torch
 import oracle
 from paper_2510_09085_b200 import workloads as W
 from tests.parity import check_hyps, masks_from_words
+from tests.refs import ctc_forward_logprob
 from tests.test_gpu_parity import _binding, _dev
 
 pytestmark = pytest.mark.gpu
@@ -140,13 +141,25 @@ def test_row_kernel_near_equal_scores_and_exact_ties():
         ln = np.array([T, T - 3, 5], dtype=np.int32)
         for K, r in [(8, 0.0), (20, 0.5), (64, 0.0)]:
             d = _run(em, ln, K, r)
-            assert d.last_call_stats()["exact_select_frames"] > 0
             res = oracle.decode(em, ln, 0, K, r, want_masks=True)
             for b in range(B):
                 check_hyps(d.hyps(b), res.hyps(b), K, max_unmatched_frac=0.3,
                            where=f"flat utt {b} K={K}", lp=em[b, : ln[b]],
                            keep=res.keep[b, : ln[b]])
             d.close()
+    # constant rows over the whole vocabulary: hundreds of candidates tie exactly, which no
+    # binning can separate - the bit-by-bit selection has to run
+    em = np.full((1, 4, 32), np.log(1.0 / 32), dtype=np.float32)
+    ln = np.array([4], dtype=np.int32)
+    d = _run(em, ln, 50, 0.0)
+    assert d.last_call_stats()["exact_select_frames"] > 0 and int(d.status[0]) == 0
+    ref = oracle.decode(em, ln, 0, 50, 0.0).hyps(0)
+    got = d.hyps(0)
+    assert len(got) == 50 and len(set(s for s, _ in got)) == 50
+    for seq, sc in got:
+        assert sc <= ctc_forward_logprob(em[0], seq, 0) + 1e-3
+    np.testing.assert_allclose(sorted(s for _, s in got), sorted(s for _, s in ref), atol=1e-3)
+    d.close()
     Tt, Vt, Kt = 5, 4, 6
     em = np.full((1, Tt, Vt), np.log(1.0 / Vt), dtype=np.float32)
     ln = np.array([Tt], dtype=np.int32)
