@@ -96,6 +96,14 @@ typedef struct {
                              sum over its alignments).  1: by max, Algorithm 1's literal
                              score' = score + logit: a prefix scores as its best alignment */
   int32_t emission_dtype; /* FLTOP_EMISSION_*: element type of the emissions */
+  int32_t max_trie_nodes; /* capacity of ONE utterance's (stream's) prefix trie, in 8-byte nodes.
+                             A node is created when a prefix enters the beam that was not in it
+                             the frame before: at most beam_width per frame.  0 = that worst
+                             case, beam_width x max_frames, which can never run out.  Peaked
+                             emissions need far less (the character workload of the benchmark:
+                             0.36 x beam_width per frame); a handle created with a smaller
+                             capacity holds less memory, and an utterance that does run out is
+                             reported with FLTOP_ST_ARENA_FULL, never written past the end */
   int32_t device;         /* CUDA device ordinal */
   void* workspace;        /* optional DEVICE memory, 256-byte aligned, for all of the
                              handle's scratch; NULL = the library allocates it */
@@ -226,7 +234,11 @@ int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t beam_width
 const char* fltop_status_string(int code);
 /* Last cudaError_t seen by this handle (0 if none). */
 int fltop_last_cuda_error(const fltop_handle* h);
-/* Bytes of beam state the handle holds: prefix trie arenas, stream states, survivor lists. */
+/* Bytes of beam state the handle holds now: prefix trie arenas, stream states and - once a
+ * call has needed them - the survivor lists of the separate prune kernel (vocabularies above
+ * 32 tokens get them at fltop_create; narrower ones only if a call cannot prune inside the
+ * decode kernel, see fltop_set_fusion, and then by a device allocation of the library's own
+ * even when the handle lives in a caller's workspace). */
 size_t fltop_beam_state_bytes(const fltop_handle* h);
 /* Kernels launched by this handle since creation. */
 int64_t fltop_launch_count(const fltop_handle* h);

@@ -33,7 +33,8 @@ class fltop_config(C.Structure):
                 ("threshold_r", C.c_float), ("max_batch", C.c_int32), ("max_frames", C.c_int32),
                 ("max_chunk_frames", C.c_int32), ("max_out_len", C.c_int32),
                 ("top_n", C.c_int32), ("beam_threshold", C.c_float), ("merge_max", C.c_int32),
-                ("emission_dtype", C.c_int32), ("device", C.c_int32),
+                ("emission_dtype", C.c_int32), ("max_trie_nodes", C.c_int32),
+                ("device", C.c_int32),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
@@ -116,10 +117,12 @@ def status_string(code: int) -> str:
 
 def make_config(vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                 max_chunk_frames=0, max_out_len=None, device=0, workspace=0, workspace_bytes=0,
-                top_n=0, beam_threshold=0.0, merge_max=0, emission_dtype=0) -> fltop_config:
+                top_n=0, beam_threshold=0.0, merge_max=0, emission_dtype=0,
+                max_trie_nodes=0) -> fltop_config:
     return fltop_config(vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                         max_chunk_frames, max_frames if max_out_len is None else max_out_len,
-                        top_n, beam_threshold, int(merge_max), int(emission_dtype), device,
+                        top_n, beam_threshold, int(merge_max), int(emission_dtype),
+                        int(max_trie_nodes), device,
                         workspace or None,
                         workspace_bytes)
 
@@ -186,11 +189,12 @@ class Decoder:
 
     def __init__(self, vocab_size, blank_id, beam_width, threshold_r, max_batch, max_frames,
                  max_chunk_frames=0, max_out_len=None, device=0, top_n=0, beam_threshold=0.0,
-                 merge_max=False, emission_dtype=torch.float32):
+                 merge_max=False, emission_dtype=torch.float32, max_trie_nodes=0):
         self.cfg = make_config(vocab_size, blank_id, beam_width, threshold_r, max_batch,
                                max_frames, max_chunk_frames, max_out_len, device, top_n=top_n,
                                beam_threshold=beam_threshold, merge_max=int(bool(merge_max)),
-                               emission_dtype=EMISSION_CODES[emission_dtype])
+                               emission_dtype=EMISSION_CODES[emission_dtype],
+                               max_trie_nodes=max_trie_nodes)
         self.emission_dtype = emission_dtype
         code, self.h = fltop_create(self.cfg)
         if code != FLTOP_OK:

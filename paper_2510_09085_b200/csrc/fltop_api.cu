@@ -44,8 +44,10 @@ struct fltop_handle {
   unsigned char* ws;
   size_t ws_bytes;
   // regions of the workspace
-  int32_t* counts;
+  int32_t* counts;        // survivor region (null until a call needs it)
   Survivor* entries;
+  unsigned char* survivor_extra;  // the region when the library allocated it by itself
+  size_t survivor_bytes, counts_bytes;
   TrieNode* nodes;
   int32_t* state;
   int32_t* stats;
@@ -89,6 +91,7 @@ bool config_ok(const fltop_config* c) {
   if (c->beam_threshold != c->beam_threshold) return false;  // NaN
   if (c->merge_max != 0 && c->merge_max != 1) return false;
   if (c->emission_dtype < FLTOP_EMISSION_F32 || c->emission_dtype > FLTOP_EMISSION_BF16) return false;
+  if (c->max_trie_nodes < 0) return false;
   if (c->device < 0) return false;
   if ((int64_t)(c->beam_width + 1) * c->max_frames + 2 > (int64_t)std::numeric_limits<int32_t>::max())
     return false;
@@ -98,25 +101,39 @@ bool config_ok(const fltop_config* c) {
 }
 
 struct Layout {
-  size_t counts, entries, nodes, state, stats, total, beam_state;
+  size_t survivors, nodes, state, stats, total, beam_state;
+  size_t survivor_bytes, counts_bytes;  // the survivor region: counts, then entries
+  bool survivors_inside;                // the region is part of the workspace
   int64_t frame_cap, nodes_per_utt;
 };
+
+// A vocabulary that the decode kernels cannot prune themselves always needs survivor lists.
+bool needs_survivor_lists(const fltop_config& c) { return c.vocab_size > 32; }
 
 Layout layout_of(const fltop_config& c) {
   Layout l;
   l.frame_cap = c.max_chunk_frames > 0 ? c.max_chunk_frames : c.max_frames;
-  // a frame takes an even-sized block of at most beam_width node ids; ids 0 and 1 are fixed
-  l.nodes_per_utt = (int64_t)((c.beam_width + 1) & ~1) * c.max_frames + 2;
+  // a frame creates at most beam_width nodes, handed out in even-sized runs; ids 0 and 1 are fixed
+  const int64_t worst = (int64_t)((c.beam_width + 1) & ~1) * c.max_frames + 2;
+  int64_t cap = worst;
+  if (c.max_trie_nodes > 0) {
+    cap = std::min<int64_t>(worst, std::max<int64_t>(c.max_trie_nodes, 2 * c.beam_width + 4));
+    cap = (cap + 1) & ~(int64_t)1;
+  }
+  l.nodes_per_utt = cap;
   const size_t frames = (size_t)c.max_batch * (size_t)l.frame_cap;
+  l.counts_bytes = up(frames * sizeof(int32_t));
+  l.survivor_bytes = l.counts_bytes + up(frames * (size_t)c.vocab_size * sizeof(Survivor));
+  l.survivors_inside = needs_survivor_lists(c);
   size_t off = 0;
-  l.counts = off; off += up(frames * sizeof(int32_t));
-  l.entries = off; off += up(frames * (size_t)c.vocab_size * sizeof(Survivor));
+  l.survivors = off;
+  if (l.survivors_inside) off += l.survivor_bytes;
   l.nodes = off; off += up((size_t)c.max_batch * (size_t)l.nodes_per_utt * sizeof(TrieNode));
   l.state = off;
   if (c.max_chunk_frames > 0) off += up((size_t)c.max_batch * state_words(c.beam_width) * 4);
-  l.beam_state = off;  // survivor lists + trie arenas + stream states
+  l.beam_state = off;  // survivor lists (if any) + trie arenas + stream states
   l.stats = off; off += up((size_t)c.max_batch * kStatWords * sizeof(int32_t));
-  l.total = off;  // survivor lists + trie arenas + stream states
+  l.total = off;
   return l;
 }
 
@@ -156,12 +173,28 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
   h->prof_valid = false;
   if (B == 0) return FLTOP_OK;
 
+  const bool fuse = h->fusion != 0 && T > 0 &&
+                    decode_can_prune(h->cfg.vocab_size, h->cfg.emission_dtype, d_logp, stride_b, stride_t);
+  if (!fuse && T > 0 && !h->counts) {
+    // the first call that needs the separate prune kernel: its survivor lists are allocated now
+    void* ptr = nullptr;
+    e = cudaMalloc(&ptr, h->survivor_bytes);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return e == cudaErrorMemoryAllocation ? FLTOP_ERR_OOM : cuda_fail(h, e);
+    }
+    h->survivor_extra = static_cast<unsigned char*>(ptr);
+    h->counts = reinterpret_cast<int32_t*>(h->survivor_extra);
+    h->entries = reinterpret_cast<Survivor*>(h->survivor_extra + h->counts_bytes);
+    h->beam_state_bytes += h->survivor_bytes;
+  }
+
   PruneParams pp;
   pp.logp = d_logp; pp.dtype = h->cfg.emission_dtype;
   pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
-  pp.counts = h->counts + (int64_t)slot0 * T;
-  pp.entries = h->entries + (int64_t)slot0 * T * h->cfg.vocab_size;
+  pp.counts = h->counts ? h->counts + (int64_t)slot0 * T : nullptr;
+  pp.entries = h->entries ? h->entries + (int64_t)slot0 * T * h->cfg.vocab_size : nullptr;
 
   DecodeParams dp = {};
   dp.lengths = d_lengths; dp.flags = d_flags; dp.B = B; dp.T = T; dp.V = h->cfg.vocab_size;
@@ -172,8 +205,6 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
   dp.merge_max = h->cfg.merge_max;
   dp.counts = pp.counts; dp.entries = pp.entries;
   dp.nodes = h->nodes + (int64_t)slot0 * h->nodes_per_utt;
-  const bool fuse = h->fusion != 0 && T > 0 &&
-                    decode_can_prune(h->cfg.vocab_size, h->cfg.emission_dtype, d_logp, stride_b, stride_t);
   dp.logp = fuse ? d_logp : nullptr; dp.dtype = h->cfg.emission_dtype;
   dp.stride_b = stride_b; dp.stride_t = stride_t;
   dp.log_r = h->log_r;
@@ -479,8 +510,12 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
     h->owns_workspace = true;
   }
   h->ws_bytes = l.total;
-  h->counts = reinterpret_cast<int32_t*>(h->ws + l.counts);
-  h->entries = reinterpret_cast<Survivor*>(h->ws + l.entries);
+  h->survivor_extra = nullptr;
+  h->survivor_bytes = l.survivor_bytes;
+  h->counts_bytes = l.counts_bytes;
+  h->counts = l.survivors_inside ? reinterpret_cast<int32_t*>(h->ws + l.survivors) : nullptr;
+  h->entries = l.survivors_inside
+                   ? reinterpret_cast<Survivor*>(h->ws + l.survivors + l.counts_bytes) : nullptr;
   h->nodes = reinterpret_cast<TrieNode*>(h->ws + l.nodes);
   h->state = cfg->max_chunk_frames > 0 ? reinterpret_cast<int32_t*>(h->ws + l.state) : nullptr;
   h->stats = reinterpret_cast<int32_t*>(h->ws + l.stats);
@@ -571,6 +606,7 @@ int fltop_destroy(fltop_handle* h) {
   for (int i = 0; i < 3; ++i)
     if (h->ev[i]) cudaEventDestroy(h->ev[i]);
   host_io_release(h->io);
+  if (h->survivor_extra && cudaFree(h->survivor_extra) != cudaSuccess) rc = FLTOP_ERR_CUDA;
   if (h->owns_workspace && h->ws && cudaFree(h->ws) != cudaSuccess) rc = FLTOP_ERR_CUDA;
   cudaGetLastError();
   delete h;
@@ -601,7 +637,10 @@ int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
   cudaError_t e = g.enter(h->cfg.device);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->last_stream);
   if (e != cudaSuccess) return cuda_fail(h, e);
-  const size_t B = (size_t)h->last_B, n_frames = B * (size_t)h->last_T;
+  const size_t B = (size_t)h->last_B;
+  // kernels that prune the frames themselves count the survivors; otherwise the prune kernel's
+  // per-frame counts are summed
+  const size_t n_frames = (h->last_fused || !h->counts) ? 0 : B * (size_t)h->last_T;
   int32_t* host = new (std::nothrow) int32_t[kStatWords * B + n_frames];
   if (!host) return FLTOP_ERR_OOM;
   e = cudaMemcpy(host, h->stats, kStatWords * B * sizeof(int32_t), cudaMemcpyDeviceToHost);
@@ -617,6 +656,7 @@ int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
       out[4] = std::max<int64_t>(out[4], s[3]);
       out[5] += s[4];
       out[6] += s[5];
+      if (h->last_fused) out[1] += s[6];
     }
     for (size_t i = 0; i < n_frames; ++i) out[1] += host[kStatWords * B + i];
   }

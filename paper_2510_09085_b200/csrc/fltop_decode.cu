@@ -1139,14 +1139,6 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     cur = nxt;
   }
   frames_seen += len;
-  if (fused()) {
-    // Survivor counts per frame are not kept (a global store in the frame loop would hold up
-    // the block's next barrier); the utterance's total stands in the first frame's place.
-    int32_t* const counts_out = p.counts + (int64_t)b * p.T;
-    for (int t1 = tid; t1 < p.T; t1 += NT) counts_out[t1] = 0;
-    __syncthreads();
-    if (tid == 0 && p.T > 0) counts_out[0] = scal[SC_KEPT];
-  }
   // the last frame's nodes; the read-out below walks the trie, so wait for all of them
   if (is_chore && lane == 0) {
     if (pend_bytes) bulk_store(nodes + pend_at, nstage + ((len - 1) & 1) * NSL, pend_bytes);
@@ -1163,6 +1155,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       int32_t* o = p.stats + kStatWords * (int64_t)b;
       o[0] = len; o[1] = scal[SC_CREATED]; o[2] = live_sum - scal[SC_DEAD]; o[3] = n_nodes;
       o[4] = scal[SC_CLASHES]; o[5] = 0;
+      o[6] = scal[SC_KEPT];  // survivors, when this kernel pruned the frames itself
     }
   }
 

@@ -978,13 +978,8 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     cur = nxt;
   }
   frames_seen += len;
-  // survivors are not listed per frame: the utterance's total stands in the first frame's place
-  {
-    int32_t* const counts_out = p.counts + (int64_t)b * p.T;
-    for (int t1 = tid; t1 < p.T; t1 += NT) counts_out[t1] = 0;
-    __syncthreads();
-    if (is_chore && lane == 0 && p.T > 0) counts_out[0] = kept_sum;
-  }
+  // (survivors are not listed per frame: their total goes out with the statistics)
+  if (p.stats && is_chore && lane == 0) p.stats[kStatWords * (int64_t)b + 6] = kept_sum;
   // the last frame's records; the read-out below walks the trie, so wait for all of them
   if (is_chore && lane == 0) {
     if (pend_bytes) bulk_store(nodes + pend_at, pend_src, pend_bytes);

@@ -451,16 +451,13 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
   frames_seen += len;
   status = (int)__reduce_or_sync(kFull, (unsigned)status);  // a lane's flag is the warp's
 
-  // survivor counts per frame are not kept: the utterance's total stands in the first place
-  {
-    int32_t* const counts_out = p.counts + (int64_t)b * p.T;
-    for (int t1 = lane; t1 < p.T; t1 += 32) counts_out[t1] = (t1 == 0) ? kept_sum : 0;
-  }
+  // (survivors are not listed per frame: their total goes out with the statistics)
   if (p.stats) {
     const int made = __reduce_add_sync(kFull, created);
     if (lane == 0) {
       int32_t* o = p.stats + kStatWords * (int64_t)b;
       o[0] = len; o[1] = made; o[2] = live_sum; o[3] = n_nodes; o[4] = 0; o[5] = 0;
+      o[6] = kept_sum;
     }
   }
 

@@ -67,8 +67,7 @@ struct DecodeParams {
   int32_t top_n;            // survivors per frame are capped at this (0: no cap)
   float beam_threshold;     // kept prefixes score at least best - beam_threshold (<= 0: off)
   int32_t merge_max;        // 1: masses are combined by max instead of log-sum
-  int32_t* counts;          // [B*T] survivors per frame (a kernel that prunes itself leaves
-                            // each utterance's total in its first frame's place, zeros after)
+  int32_t* counts;          // [B*T] survivors per frame (not touched by a kernel that prunes itself)
   const Survivor* entries;  // [B*T*V]
   // Non-null: the decode kernel prunes the rows itself (V <= 32) and `entries` is not read.
   const void* logp;         // elements of `dtype`
@@ -92,7 +91,9 @@ struct DecodeParams {
   int32_t dbg_frame0, dbg_frames;
 };
 // per-utterance statistics of a call: frames, trie nodes created, sum of beam sizes, node ids
-// used, fingerprint-tag clashes (probes that met another sequence with the same 20-bit tag)
+// used, fingerprint-tag clashes (probes that met another sequence with the same 20-bit tag),
+// frames selected by the slow exact path, survivors over all frames (kernels that prune
+// the frames themselves; the others leave the per-frame counts of the prune kernel)
 constexpr int kStatWords = 8;
 
 size_t decode_smem_bytes(int K, int V);

@@ -40,7 +40,7 @@ def test_config_struct_matches_header(bd):
     dict(vocab_size=1), dict(vocab_size=9000), dict(blank_id=-1), dict(blank_id=32),
     dict(beam_width=0), dict(beam_width=5000), dict(threshold_r=-0.1), dict(threshold_r=1.5),
     dict(threshold_r=float("nan")), dict(max_batch=0), dict(max_frames=0), dict(max_out_len=0),
-    dict(top_n=-1), dict(beam_threshold=float("nan")), dict(merge_max=2), dict(emission_dtype=3), dict(emission_dtype=-1), dict(device=-1), dict(max_chunk_frames=-1),
+    dict(top_n=-1), dict(max_trie_nodes=-1), dict(beam_threshold=float("nan")), dict(merge_max=2), dict(emission_dtype=3), dict(emission_dtype=-1), dict(device=-1), dict(max_chunk_frames=-1),
     dict(max_chunk_frames=101), dict(workspace=8, workspace_bytes=1 << 40),
     dict(beam_width=2048, vocab_size=8192),     # needs more shared memory than one SM has
 ])
@@ -80,14 +80,27 @@ def test_null_arguments(bd):
 
 
 def test_workspace_size_accounts_for_every_region(bd):
+    # a character vocabulary is pruned inside the decode kernel: no survivor lists in the
+    # workspace, only the trie arenas (8-byte nodes) and the per-utterance statistics
     cfg = bd.make_config(32, 0, 50, 1e-3, 64, 1750)
     need = bd.fltop_workspace_size(cfg)
-    frames = 64 * 1750
-    expect = frames * 4 + frames * 32 * 8 + 64 * (50 * 1750 + 2) * 8  # counts, survivors, 8-byte trie nodes
-    assert expect <= need <= expect + 4 * 256 + 64 * 32  # + per-utterance statistics
+    expect = 64 * (50 * 1750 + 2) * 8
+    assert expect <= need <= expect + 2 * 256 + 64 * 32
+    # a smaller trie capacity shrinks it; it is never taken below what two frames can create
+    small = bd.make_config(32, 0, 50, 1e-3, 64, 1750, max_trie_nodes=40000)
+    assert 64 * 40000 * 8 <= bd.fltop_workspace_size(small) <= 64 * 40000 * 8 + 2 * 256 + 64 * 32
+    tiny = bd.make_config(32, 0, 50, 1e-3, 64, 1750, max_trie_nodes=1)
+    assert bd.fltop_workspace_size(tiny) >= 64 * (2 * 50 + 4) * 8
+    huge = bd.make_config(32, 0, 50, 1e-3, 64, 1750, max_trie_nodes=2 ** 31 - 1)
+    assert bd.fltop_workspace_size(huge) == need
+    # wider vocabularies take the separate prune kernel: counts and survivor lists are inside
+    frames = 8 * 100
+    wide = bd.make_config(1024, 0, 8, 1e-3, 8, 100)
+    expect = frames * 4 + frames * 1024 * 8 + 8 * (8 * 100 + 2) * 8
+    assert expect <= bd.fltop_workspace_size(wide) <= expect + 4 * 256 + 8 * 32
     scfg = bd.make_config(32, 0, 16, 1e-2, 1024, 1600, max_chunk_frames=16)
     sneed = bd.fltop_workspace_size(scfg)
-    assert sneed < 1024 * (16 * 1600 + 2) * 8 + 1024 * 16 * (4 + 256) + 1024 * 4 * 200 + 4096
+    assert sneed < 1024 * (16 * 1600 + 2) * 8 + 1024 * 4 * 200 + 64 * 1024
     too_small = bd.make_config(32, 0, 50, 1e-3, 64, 1750, workspace=256, workspace_bytes=1024)
     assert bd.fltop_create(too_small)[0] == bd.FLTOP_ERR_OOM
 

@@ -236,3 +236,34 @@ def test_block_kernel_with_fewer_stay_lanes_than_beam_entries():
     for i, b in enumerate(sample):
         check_hyps(d.hyps(b), res.hyps(i), K, where=f"utt {b}")
     d.close()
+
+
+def test_trie_capacity_knob_and_lazy_survivor_lists():
+    # max_trie_nodes: a capacity below the worst case holds less memory and changes nothing as
+    # long as it suffices; one that runs out is reported per utterance, never written past
+    bd = _binding()
+    wl = W.workload_wav2vec2(batch=8)
+    B, T, V = wl.emissions.shape
+    K, r = 50, 1e-3
+    full = _run(wl.emissions, wl.lengths, K, r)
+    used = full.last_call_stats()["max_node_ids_used"]
+    assert used < 0.5 * K * T
+    half = _run(wl.emissions, wl.lengths, K, r, max_trie_nodes=K * T // 2)
+    assert half.beam_state_bytes < 0.55 * full.beam_state_bytes
+    assert (half.status[:B] == 0).all()
+    for b in range(B):
+        assert half.hyps(b) == full.hyps(b)
+    short = _run(wl.emissions, wl.lengths, K, r, max_trie_nodes=used // 2)
+    st = short.status.cpu().numpy()[:B]
+    assert (st & bd.FLTOP_ST_ARENA_FULL).any() and not (st & ~bd.FLTOP_ST_ARENA_FULL).any()
+    assert (short.lens.cpu().numpy()[:B] <= T).all()
+    # survivor lists exist only once a call takes the separate prune kernel
+    before = half.beam_state_bytes
+    half.set_fusion(0)
+    half.decode(_dev(wl.emissions), _dev(wl.lengths))
+    torch.cuda.synchronize()
+    assert half.beam_state_bytes >= before + B * T * V * 8
+    for b in range(B):
+        _same_hyps(half.hyps(b), full.hyps(b), f"utt {b}")
+    for d in (full, half, short):
+        d.close()
