@@ -37,9 +37,36 @@ UNIT = "frames/s"
 BATCH, BEAM, R_PRUNED = 64, 50, 1e-3
 L2_FLUSH_BYTES = 256 << 20
 NODE_BYTES, SURVIVOR_BYTES = 8, 8
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch on the default workload
-# (profiles/decode_kernel_wav2vec2_B64_K50_full.txt); None whenever the kernel has changed since
-DECODE_DRAM_BYTES = 7.47e6
+# ncu's DRAM byte count of one launch of the dominant kernel on the default workload is kept
+# beside its profile summary, together with a hash of the kernel's sources: the bench reports
+# it as `roofline.traffic` only while the sources still are the ones that were profiled
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "decode_rows_kernel_wav2vec2_B64_K50_full.txt")
+KERNEL_SOURCES = ("fltop_decode_rows.cu", "fltop_device.cuh", "fltop_internal.h")
+
+
+def kernel_source_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2510_09085_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic():
+    """DRAM bytes per launch from the profile summary, or None if the kernel changed since."""
+    try:
+        text = open(TRAFFIC_RECORD).read()
+    except OSError:
+        return None
+    rec = dict(line.split(":", 1) for line in text.splitlines()
+               if line.startswith(("dram_bytes_per_launch:", "kernel_source_hash:")))
+    if rec.get("kernel_source_hash", "").strip() != kernel_source_hash():
+        return None
+    try:
+        return float(rec["dram_bytes_per_launch"])
+    except (KeyError, ValueError):
+        return None
 
 
 def _algorithmic_bytes(V, st, out_bytes, fused, esize=4):
@@ -48,10 +75,9 @@ def _algorithmic_bytes(V, st, out_bytes, fused, esize=4):
     Two kernels: the prune kernel reads every emission row and writes a count and the survivor
     list per frame, the decode kernel reads those back.  One kernel (it prunes its own rows):
     the emission rows are the decode kernel's input and no survivor list exists.  Either way
-    the decode kernel writes one block of 8-byte trie records per frame (one record per beam
-    slot, rounded up to an even count) and the hypotheses at the end.  ``esize``: bytes per
-    stored emission (4, or 2 for fp16 / bf16)."""
-    trie = NODE_BYTES * (st["live_hypotheses_sum"] + st["frames"])
+    the decode kernel writes one 8-byte trie record per prefix that enters the beam and the
+    hypotheses at the end.  ``esize``: bytes per stored emission (4, or 2 for fp16 / bf16)."""
+    trie = NODE_BYTES * st["trie_nodes_created"]
     if fused:
         return 0, st["frames"] * esize * V + trie + out_bytes
     prune = st["frames"] * (esize * V + 4) + st["survivors"] * SURVIVOR_BYTES
@@ -227,7 +253,11 @@ def run_ours(args):
     stream = torch.cuda.Stream()
 
     def make(r):
-        d = binding.Decoder(V, wl.blank_id, BEAM, r, B, T, device=local_rank)
+        # trie capacity: half the worst case of one new prefix per beam slot and frame (the
+        # workload creates 0.36 per slot and frame; running out would be reported per utterance
+        # and is asserted not to happen below)
+        d = binding.Decoder(V, wl.blank_id, BEAM, r, B, T, device=local_rank,
+                            max_trie_nodes=max(1024, BEAM * T // 2))
         d.set_profiling(True)
         return d
 
@@ -320,18 +350,25 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_p,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": wl.name, "batch_per_gpu": B, "beam": BEAM, "r": R_PRUNED,
-                   "vocab": V, "frames_per_step_per_gpu": n_frames, "max_frames": int(T),
+        "config": {"workload": wl.name if world == 1 else f"{wl.name} (rank 0's share)",
+                   "utterances": n_global, "utterances_rank0": B, "beam": BEAM, "r": R_PRUNED,
+                   "vocab": V, "frames_per_step_rank0": n_frames, "max_frames": int(T),
                    "l2": f"flushed: {L2_FLUSH_BYTES >> 20} MiB written between timed steps",
-                   "sharding": "one independent batch per GPU, no collective"},
+                   "sharding": ("every GPU draws its own batch of 64 utterances" if args.independent
+                                else "one batch of 64 utterances per GPU, split over the GPUs by total "
+                                     "frames, longest first; no collective on the data path")},
         "e2e": {"value": value_e, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": t_e,
                 "call": "fltop_decode_host: pinned host emissions in, host hypotheses out; "
                         "the valid frames and the existing tokens are what crosses the bus"},
         "gpu_launches": launches,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved,
-                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": (DECODE_DRAM_BYTES if args.workload == "wav2vec2" and not args.batch else None),
+        "roofline": {"bound": "hbm",
+                     "kernel": "decode_rows_kernel" if V <= 32 and BEAM <= 64 else "decode_kernel",
+                     "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": (recorded_traffic() if args.workload == "wav2vec2" and not args.batch
+                                 and world == 1 else None),
                      "peak_source": f"{peak_kind} copy bandwidth",
                      "bytes_per_launch": db, "ms_per_launch": dk_ms,
                      "note": "latency-bound serial frame chain: max_frames dependent steps"},
@@ -344,7 +381,7 @@ def run_ours(args):
                    "mean_live_hypotheses": stats_0["live_hypotheses_sum"] / max(1, stats_0["frames"]),
                    "hbm_frac_step": (pb0 + db0) / (t_0 * 1e-3) / 1e9 / peak},
             "pruned_over_r0_speedup": t_0 / t_p,
-            "utterances_per_s": world * B / (t_p * 1e-3),
+            "utterances_per_s": n_global / (t_p * 1e-3),
             "prune_kernel_ms": statistics.mean(prune_p),
             "decode_kernel_ms": dk_ms,
             "ns_per_frame_step": 1e6 * dk_ms / int(wl.lengths.max()),
@@ -356,6 +393,7 @@ def run_ours(args):
                                  if statistics.mean(prune_p) > 0 else None),
             "pruning": "inside the decode kernel" if launches_per_step == 1 else "separate kernel",
             "beam_state_bytes": dec_p.beam_state_bytes,
+            "beam_state_bytes_written": NODE_BYTES * stats_p["trie_nodes_created"],
             "step_ms_min": min(ms_p), "step_ms_median": statistics.median(ms_p),
         },
     }

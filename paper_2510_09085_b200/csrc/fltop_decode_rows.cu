@@ -372,7 +372,11 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   // Chore warp: what the warps need to know about frame t1 (its row has landed).  One token
   // per lane: row maximum by a warp reduction, the relative threshold by one float32 add and
   // compare (Algorithm 1's conditional break), the survivors by a ballot.
-  auto prepare = [&](int t1) {
+  // In two halves, so that each fits into a stretch in which the chore warp has nothing else
+  // to do: the first ends with the survivor set, the second lays the survivors out.
+  float prep_v = neg_inf();   // (chore warp) the row being prepared, one token per lane
+  unsigned prep_kept = 0u;    // ... and its survivors
+  auto prepare_survivors = [&](int t1) {
     float v = neg_inf();
     if (p.dtype == kEmissionF32) {
       if (lane < V) v = S.raw[t1 & 3][lane];
@@ -401,6 +405,12 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
       }
       kept = chosen;
     }
+    prep_v = v;
+    prep_kept = kept;
+  };
+  auto prepare_layout = [&](int t1) {
+    const float v = prep_v;
+    const unsigned kept = prep_kept;
     const float lb = __shfl_sync(kFull, v, blank);
     const unsigned kept_nb = kept & ~(1u << blank);
     const int snb = __popc(kept_nb);
@@ -418,6 +428,10 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
       kept_sum += __popc(kept);
       if ((HOOKS & 1) && p.dbg_masks) p.dbg_masks[(int64_t)b * p.T + t1] = kept;
     }
+  };
+  auto prepare = [&](int t1) {
+    prepare_survivors(t1);
+    prepare_layout(t1);
   };
   if (is_chore) {
     if (len > 0) fetch_row(0);
@@ -452,6 +466,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
       cp_async_commit();
       cp_async_wait_but_one();  // the row requested a frame ago has landed
       __syncwarp();
+      if (t + 2 < len) prepare_survivors(t + 2);
     };
     // A frame in which only blank survives (Algorithm 1's conditional break has dropped every
     // other token): every prefix stays, by blank, and nothing is selected, merged or created.
@@ -466,7 +481,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         S.hot[cur][tid] = e;
       } else if (is_chore) {
         chore_window();
-        if (t + 2 < len) prepare(t + 2);
+        if (t + 2 < len) prepare_layout(t + 2);
       }
       drift += head.lp_blank;
       pend_bytes = 0u;
@@ -738,9 +753,9 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
       reinterpret_cast<uint4*>(hist)[lane + 32] = zero;
       if (lane < KMAX / 4) reinterpret_cast<uint4*>(S.dupw[par ^ 1])[lane] = zero;
       if (lane < FS_COUNT) S.fs[par ^ 1][lane] = 0;
-      // frame t+2 as the warps will see it (its row has landed; the buffers it goes into were
-      // last read in frame t-2)
-      if (t + 2 < len) prepare(t + 2);
+      // frame t+2 as the warps will see it (the buffers it goes into were last read in
+      // frame t-2); the survivor set was worked out while the others evaluated
+      if (t + 2 < len) prepare_layout(t + 2);
     };
 
     if (n_listed <= kListCap) {
@@ -1089,8 +1104,12 @@ int decode_rows_threads(const DecodeParams& p, bool alone) {
   if (p.top_n > 0 && p.top_n < cols) cols = p.top_n;
   const int per_row = p.K >= 32 ? 1 : 32 / (p.K <= 1 ? 1 : 1 << (32 - __builtin_clz(p.K - 1)));
   const int rows = (cols + per_row - 1) / per_row;   // token rows of a frame
-  int P = alone ? (rows + 1) / 2 : (rows + 3) / 4;   // two / four token rows per warp
+  // measured on B200 (64 utterances, V = 32): with pruning on four warps per block of beam
+  // entries for beams above 32, six below; without, as many as fit; a quarter of that when
+  // blocks share SMs
+  int P = alone ? (rows + 1) / 2 : (rows + 3) / 4;
   const int cap = ((alone ? 16 : 8) - 1 - nsw) / nsw;
+  if (alone && p.pruning && nsw > 1 && P > 4) P = 4;
   if (P > cap) P = cap;
   if (P < 1) P = 1;
   return 32 * (nsw + 1 + nsw * P);
