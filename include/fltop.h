@@ -210,8 +210,11 @@ int fltop_prune(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t s
  *     rounded up to an even number; anything
  *     larger returns FLTOP_ERR_CAPACITY and launches nothing;
  *   - it runs on the CURRENT device.  The first call on each device looks up the array's
- *     device address (cudaGetSymbolAddress) before launching; make that first call outside
- *     any stream capture;
+ *     device address (cudaGetSymbolAddress) and sets the decode kernel's launch attributes
+ *     before launching (the latter again for a shape that needs another layout of the
+ *     kernel); the driver may load the kernels and the array onto the device at that point.
+ *     Make that first call - a warm-up - outside any stream capture and outside any
+ *     real-time section;
  *   - all calls share the one array.  It needs no clearing between calls (every word a
  *     call reads it has written first), but two calls whose kernels overlap on the GPU -
  *     different streams, or different host threads - race on it.  Serialise them.

@@ -107,8 +107,9 @@ struct Layout {
   int64_t frame_cap, nodes_per_utt;
 };
 
-// A vocabulary that the decode kernels cannot prune themselves always needs survivor lists.
-bool needs_survivor_lists(const fltop_config& c) { return c.vocab_size > 32; }
+// A vocabulary that the decode kernels cannot prune themselves always needs survivor lists
+// (narrower ones get them on the first call that cannot be pruned inside, if ever).
+bool needs_survivor_lists(const fltop_config& c) { return c.vocab_size > 1024; }
 
 Layout layout_of(const fltop_config& c) {
   Layout l;
@@ -174,7 +175,8 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
   if (B == 0) return FLTOP_OK;
 
   const bool fuse = h->fusion != 0 && T > 0 &&
-                    decode_can_prune(h->cfg.vocab_size, h->cfg.emission_dtype, d_logp, stride_b, stride_t);
+                    decode_can_prune(h->cfg.vocab_size, h->cfg.emission_dtype, d_logp, stride_b, stride_t,
+                                     h->cfg.top_n);
   if (!fuse && T > 0 && !h->counts) {
     // the first call that needs the separate prune kernel: its survivor lists are allocated now
     void* ptr = nullptr;

@@ -76,6 +76,10 @@ __device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) 
   const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(d), "l"(gmem_src));
 }
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src));
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n"); }
 __device__ __forceinline__ void cp_async_wait_all() {
   asm volatile("cp.async.wait_group 0;\n" ::: "memory");
@@ -156,6 +160,11 @@ __host__ __device__ inline int node_stage_len(int K) { return (K + 1) & ~1; }
 // Byte offsets of the shared-memory arrays.
 // widest vocabulary whose frames the decode block prunes itself (one token per lane)
 constexpr int kFusedMaxV = 32;
+// ... and the widest whose frames it prunes itself with the chore warp walking the row
+constexpr int kFusedWideMaxV = 1024;
+__host__ __device__ inline int raw_row_len(int V) {
+  return (V > kFusedMaxV && V <= kFusedWideMaxV) ? V : kFusedMaxV;
+}
 // up to this many stay lanes, every stay warp looks at all stay candidates itself (P3a)
 constexpr int kOwnStayLanes = 128;
 
@@ -173,7 +182,7 @@ __host__ __device__ inline Lay make_layout(int K, int V) {
     off += (bytes + 15u) & ~15u;
     return at;
   };
-  l.raw = take(4u * kFusedMaxV * 4);  // first: its address needs no offset
+  l.raw = take(4u * raw_row_len(V) * 4);  // first: its address needs no offset
   l.sv = take(4u * V * 8);
   l.hot = take(2u * K * 16);
   l.ident = take(2u * K * 16);
@@ -483,20 +492,53 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   // (Nothing of this is kept in registers across the frame loop: the large blocks have 64 a
   // thread, and every thread would pay for what only the chore warp uses.)
   auto fused = [&]() -> bool { return p.logp != nullptr; };
+  const int RS = raw_row_len(VS);  // floats between the raw rows of consecutive frames
   auto raw_row = [&](int t1) -> float* {
-    return reinterpret_cast<float*>(smem) + (t1 & 3) * kFusedMaxV;
+    return reinterpret_cast<float*>(smem) + (t1 & 3) * RS;
   };
   // float32 rows: a word per lane; fp16 / bf16 rows: a word holds two tokens (V is even then)
   auto fetch_row = [&](int t1) {
     const int64_t at = (int64_t)b * p.stride_b + (int64_t)t1 * p.stride_t;
-    if (p.dtype == kEmissionF32) {
+    if (V > kFusedMaxV) {
+      // a wide row (float32, 16-byte aligned, V a multiple of four): 16 bytes per lane and turn
+      const float* src = static_cast<const float*>(p.logp) + at;
+      for (int c = 4 * lane; c < V; c += 128) cp_async16(raw_row(t1) + c, src + c);
+    } else if (p.dtype == kEmissionF32) {
       if (lane < V) cp_async4(raw_row(t1) + lane, static_cast<const float*>(p.logp) + at + lane);
     } else if (2 * lane < V) {
       cp_async4(raw_row(t1) + lane, static_cast<const uint16_t*>(p.logp) + at + 2 * lane);
     }
   };
   // the row of frame t1 has landed; returns the survivor count
+  // order-preserving integer key of a float32 (a NaN sorts below every number)
+  auto okey = [](float v) -> unsigned {
+    const unsigned vu = __float_as_uint(v);
+    return (v == v) ? ((vu & 0x80000000u) ? ~vu : (vu | 0x80000000u)) : 0x007fffffu;
+  };
+  // a row of more than 32 tokens: the chore warp walks it twice, 32 tokens a turn - the row
+  // maximum, then the survivors in ascending token order
+  auto prune_wide_row = [&](int t1) -> int {
+    const float* const row = raw_row(t1);
+    unsigned key = 0u;
+    for (int c = lane; c < V; c += 32) key = max(key, okey(row[c]));
+    const unsigned mkey = __reduce_max_sync(kFull, key);
+    const float m = __uint_as_float((mkey & 0x80000000u) ? (mkey & 0x7fffffffu) : ~mkey);
+    const float thr = __fadd_rn(m, p.log_r);
+    Survivor* const out = svbuf(t1);
+    int n = 0;
+    for (int c0 = 0; c0 < V; c0 += 32) {
+      const int c = c0 + lane;
+      const float v = c < V ? row[c] : neg_inf();
+      const bool keep = c < V && v >= thr;
+      const unsigned kept = __ballot_sync(kFull, keep);
+      if (keep) out[n + __popc(kept & lt_mask)] = Survivor{c, v};
+      n += __popc(kept);
+    }
+    if (lane == 0) scal[SC_KEPT] += n;
+    return n;
+  };
   auto prune_row = [&](int t1) -> int {
+    if (V > kFusedMaxV) return prune_wide_row(t1);
     float v = neg_inf();
     if (p.dtype == kEmissionF32) {
       if (lane < V) v = raw_row(t1)[lane];  // the word this lane fetched itself
@@ -1301,8 +1343,15 @@ void launch_variant(const DecodeParams& p, int nt, size_t bytes, bool alone, cud
 }
 }  // namespace
 
-bool decode_can_prune(int V, int dtype, const void* logp, int64_t stride_b, int64_t stride_t) {
-  if (V > kFusedMaxV) return false;
+bool decode_can_prune(int V, int dtype, const void* logp, int64_t stride_b, int64_t stride_t,
+                      int top_n) {
+  if (V > kFusedWideMaxV) return false;
+  if (V > kFusedMaxV) {
+    // wide rows are fetched 16 bytes at a time and walked by one warp: float32, rows that
+    // start on a 16-byte boundary, no top-N stage (that is the cap kernel's radix select)
+    return dtype == kEmissionF32 && (top_n <= 0 || top_n >= V) && V % 4 == 0 &&
+           stride_b % 4 == 0 && stride_t % 4 == 0 && (reinterpret_cast<uintptr_t>(logp) & 15u) == 0;
+  }
   if (dtype == kEmissionF32) return true;
   // two-byte elements are fetched in pairs: every row has to start on a four-byte boundary
   return V % 2 == 0 && stride_b % 2 == 0 && stride_t % 2 == 0 &&

@@ -110,6 +110,7 @@ bool decode_warp_eligible(const DecodeParams& p);
 cudaError_t launch_decode_warp(const DecodeParams& p, cudaStream_t s);
 cudaError_t decode_prepare(int K, int V);  // one-time kernel attribute set-up
 // the decode kernel can take these raw emission rows itself (strides in elements)
-bool decode_can_prune(int V, int dtype, const void* logp, int64_t stride_b, int64_t stride_t);
+bool decode_can_prune(int V, int dtype, const void* logp, int64_t stride_b, int64_t stride_t,
+                      int top_n);
 
 }  // namespace fltop

@@ -38,15 +38,28 @@ static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 constexpr int kMaxDevices = 64;
 std::mutex g_setup_lock;
 unsigned char* g_scratch_addr[kMaxDevices] = {nullptr};
+// fixed layouts of the decode kernel whose launch attributes are set on a device (bits)
+unsigned g_prepared[kMaxDevices] = {0u};
 
-// Device address of the scratch on the current device (first call per device sets it up).
-cudaError_t scratch_address(int device, unsigned char** out) {
+// Device address of the scratch on the current device, and the decode kernel ready to be
+// launched for this beam width and vocabulary.  The first call per device (and per layout
+// variant of the kernel) does the set-up: it may load the kernels and the array onto the
+// device, so it belongs outside stream capture and outside real-time sections.
+cudaError_t set_up(int device, int K, int V, unsigned char** out) {
   std::lock_guard<std::mutex> guard(g_setup_lock);
   if (!g_scratch_addr[device]) {
     void* ptr = nullptr;
     const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
     if (e != cudaSuccess) return e;
     g_scratch_addr[device] = static_cast<unsigned char*>(ptr);
+  }
+  // Beams of at most 64 use one of two fixed layouts (vocabulary up to 32, or wider); their
+  // attributes are set once.  Wider beams size their shared memory by the beam itself.
+  const unsigned variant = K <= 64 ? (V <= 32 ? 1u : 2u) : 0u;
+  if (variant == 0u || !(g_prepared[device] & variant)) {
+    const cudaError_t e = decode_prepare(K, V);
+    if (e != cudaSuccess) return e;
+    g_prepared[device] |= variant;
   }
   *out = g_scratch_addr[device];
   return cudaSuccess;
@@ -68,7 +81,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   if (!d_lengths || !d_tokens || !d_lens || !d_scores || !d_nhyp) return FLTOP_ERR_INVALID_ARG;
   if (T > 0 && (!d_logp || stride_t < vocab_size || stride_b < 0)) return FLTOP_ERR_INVALID_ARG;
   // the fixed scratch bounds the problem size
-  const int64_t nodes_per_utt = (int64_t)((beam_width + 1) & ~1) * (T > 0 ? T : 1) + 2;
+  const int64_t nodes_per_utt = (int64_t)((beam_width + 1) & ~1) * T + 2;
   if (vocab_size > kStaticMaxVocab || (int64_t)B * T > kStaticMaxFrames ||
       (int64_t)B * nodes_per_utt > kStaticMaxNodes)
     return FLTOP_ERR_CAPACITY;
@@ -78,8 +91,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   cudaError_t e = cudaGetDevice(&device);
   if (e != cudaSuccess || device >= kMaxDevices) { cudaGetLastError(); return FLTOP_ERR_CUDA; }
   unsigned char* scratch = nullptr;
-  e = scratch_address(device, &scratch);
-  if (e == cudaSuccess) e = decode_prepare(beam_width, vocab_size);
+  e = set_up(device, beam_width, vocab_size, &scratch);
   if (e != cudaSuccess) { cudaGetLastError(); return FLTOP_ERR_CUDA; }
 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

@@ -93,10 +93,11 @@ def test_workspace_size_accounts_for_every_region(bd):
     assert bd.fltop_workspace_size(tiny) >= 64 * (2 * 50 + 4) * 8
     huge = bd.make_config(32, 0, 50, 1e-3, 64, 1750, max_trie_nodes=2 ** 31 - 1)
     assert bd.fltop_workspace_size(huge) == need
-    # wider vocabularies take the separate prune kernel: counts and survivor lists are inside
+    # vocabularies above 1024 always take the separate prune kernel: counts and survivor
+    # lists are inside
     frames = 8 * 100
-    wide = bd.make_config(1024, 0, 8, 1e-3, 8, 100)
-    expect = frames * 4 + frames * 1024 * 8 + 8 * (8 * 100 + 2) * 8
+    wide = bd.make_config(2048, 0, 8, 1e-3, 8, 100)
+    expect = frames * 4 + frames * 2048 * 8 + 8 * (8 * 100 + 2) * 8
     assert expect <= bd.fltop_workspace_size(wide) <= expect + 4 * 256 + 8 * 32
     scfg = bd.make_config(32, 0, 16, 1e-2, 1024, 1600, max_chunk_frames=16)
     sneed = bd.fltop_workspace_size(scfg)

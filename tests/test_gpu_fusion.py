@@ -160,13 +160,57 @@ def test_fused_streaming_equals_one_shot(C):
     one.close()
 
 
-def test_wide_vocabularies_keep_the_separate_kernel():
-    em, ln = W.make_small(81, 2, 20, 20, 48)
-    d, launches = _decode(_dev(em), ln, 48, 8, 1e-2, 1)
+@pytest.mark.parametrize("V,K,r", [(48, 8, 1e-2), (64, 50, 1e-3), (300, 4, 0.05), (1024, 32, 1e-3),
+                                   (1024, 32, 0.0), (1024, 100, 1e-3), (256, 300, 1e-2)])
+def test_fused_pruning_of_wide_rows_changes_nothing(V, K, r):
+    # vocabularies of 33 to 1024 tokens: the decode block walks its own rows (float32, rows on
+    # 16-byte boundaries, no top-N stage); bit for bit what the separate prune kernel gives
+    B = 6
+    em, ln = W.make_small(8100 + V + K, B, 40, 40, V)
+    T = em.shape[1]
+    ln[:5] = [0, 1, 2, 3, T]
+    em[:, :, :] = np.where(np.arange(T)[None, :, None] < ln[:, None, None], em, np.nan)
+    x = _dev(em)
+    fused, n_fused = _decode(x, ln, V, K, r, 1)
+    apart, n_apart = _decode(x, ln, V, K, r, 0)
+    assert n_fused == 1 and n_apart == 2
+    assert (fused.status[:B] == 0).all()
+    _same_outputs(fused, apart, B)
+    clean = np.nan_to_num(em, nan=0.0)
+    res = oracle.decode(clean, ln, 0, K, r, want_masks=True)
+    for b in range(B):
+        check_hyps(fused.hyps(b), res.hyps(b), K, where=f"V={V} utt {b}", lp=clean[b, : ln[b]],
+                   keep=res.keep[b, : ln[b]], max_unmatched_frac=0.25 if K >= 100 else 0.0)
+    assert fused.beam_state_bytes < apart.beam_state_bytes      # no survivor lists
+    fused.close()
+    apart.close()
+
+
+def test_rows_that_cannot_be_pruned_inside_take_the_separate_kernel():
+    # a vocabulary that is not a multiple of four, rows off the 16-byte grid, a top-N stage on a
+    # wide vocabulary, more than 1024 tokens: two (or three) launches, same results as ever
+    em, ln = W.make_small(81, 2, 20, 20, 50)
+    d, launches = _decode(_dev(em), ln, 50, 8, 1e-2, 1)
     assert launches == 2
     res = oracle.decode(em, ln, 0, 8, 1e-2)
     for b in range(2):
-        check_hyps(d.hyps(b), res.hyps(b), 8, where=f"V=48 utt {b}")
+        check_hyps(d.hyps(b), res.hyps(b), 8, where=f"V=50 utt {b}")
+    d.close()
+    em, ln = W.make_small(82, 2, 20, 20, 64)
+    wide = torch.zeros((2, 20, 70), device="cuda")
+    wide[:, :, 3:67] = _dev(em)
+    d, launches = _decode(wide[:, :, 3:67], ln, 64, 8, 1e-2, 1)
+    assert launches == 2
+    d.close()
+    d, launches = _decode(_dev(em), ln, 64, 8, 1e-2, 1, top_n=4)
+    assert launches == 3
+    res = oracle.decode(em, ln, 0, 8, 1e-2, top_n=4)
+    for b in range(2):
+        check_hyps(d.hyps(b), res.hyps(b), 8, where=f"V=64 top-4 utt {b}")
+    d.close()
+    em, ln = W.make_small(83, 2, 12, 12, 2048)
+    d, launches = _decode(_dev(em), ln, 2048, 8, 1e-3, 1)
+    assert launches == 2
     d.close()
 
 
