@@ -515,25 +515,47 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     const unsigned vu = __float_as_uint(v);
     return (v == v) ? ((vu & 0x80000000u) ? ~vu : (vu | 0x80000000u)) : 0x007fffffu;
   };
-  // a row of more than 32 tokens: the chore warp walks it twice, 32 tokens a turn - the row
-  // maximum, then the survivors in ascending token order
-  auto prune_wide_row = [&](int t1) -> int {
-    const float* const row = raw_row(t1);
-    unsigned key = 0u;
-    for (int c = lane; c < V; c += 32) key = max(key, okey(row[c]));
-    const unsigned mkey = __reduce_max_sync(kFull, key);
-    const float m = __uint_as_float((mkey & 0x80000000u) ? (mkey & 0x7fffffffu) : ~mkey);
-    const float thr = __fadd_rn(m, p.log_r);
-    Survivor* const out = svbuf(t1);
-    int n = 0;
-    for (int c0 = 0; c0 < V; c0 += 32) {
-      const int c = c0 + lane;
-      const float v = c < V ? row[c] : neg_inf();
-      const bool keep = c < V && v >= thr;
-      const unsigned kept = __ballot_sync(kFull, keep);
-      if (keep) out[n + __popc(kept & lt_mask)] = Survivor{c, v};
-      n += __popc(kept);
+  // A row of more than 32 tokens (V a multiple of four): the chore warp walks it twice, four
+  // tokens per lane and turn - first the row maximum and with it the threshold, then the
+  // survivors in ascending token order.  The two walks are separate calls: within the frame
+  // loop each takes a stretch in which the chore warp would otherwise wait.
+  auto wide_row_threshold = [&](int t1) -> float {
+    const float4* const row = reinterpret_cast<const float4*>(raw_row(t1));
+    float m = neg_inf();
+    for (int c = lane; 4 * c < V; c += 32) {
+      const float4 x = row[c];
+      m = fmaxf(m, fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w)));  // (a NaN never is the maximum)
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, o));
+    return __fadd_rn(m, p.log_r);
+  };
+  // (tokens [4 * from, 4 * to) of the row, appended to the n survivors found so far)
+  auto wide_row_survivors = [&](int t1, float thr, int from, int to, int n) -> int {
+    const float4* const row = reinterpret_cast<const float4*>(raw_row(t1));
+    Survivor* const out = svbuf(t1);
+    for (int c0 = from; c0 < to; c0 += 32) {
+      const int c = c0 + lane;
+      const bool in = c < to;
+      const float4 x = in ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      const bool k0 = in && x.x >= thr, k1 = in && x.y >= thr, k2 = in && x.z >= thr,
+                 k3 = in && x.w >= thr;
+      const unsigned b0 = __ballot_sync(kFull, k0), b1 = __ballot_sync(kFull, k1),
+                     b2 = __ballot_sync(kFull, k2), b3 = __ballot_sync(kFull, k3);
+      // tokens 4c .. 4c+3 of lane c come after everything the lanes before it keep
+      int at = n + __popc(b0 & lt_mask) + __popc(b1 & lt_mask) + __popc(b2 & lt_mask) +
+               __popc(b3 & lt_mask);
+      if (k0) out[at++] = Survivor{4 * c, x.x};
+      if (k1) out[at++] = Survivor{4 * c + 1, x.y};
+      if (k2) out[at++] = Survivor{4 * c + 2, x.z};
+      if (k3) out[at++] = Survivor{4 * c + 3, x.w};
+      n += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+    }
+    return n;
+  };
+  const int wide_half = ((V / 4 + 63) / 64) * 32;  // float4s of the first half of a wide row
+  auto prune_wide_row = [&](int t1) -> int {
+    const int n = wide_row_survivors(t1, wide_row_threshold(t1), 0, V / 4, 0);
     if (lane == 0) scal[SC_KEPT] += n;
     return n;
   };
@@ -727,6 +749,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       if (lane < SC_PER_FRAME) scal[(par ^ 1) * SC_PER_FRAME + lane] = 0;
     };
     // ---- P1: every candidate is evaluated once and counted -----------------------------
+    float wide_thr = neg_inf();  // (chore warp, wide rows) the threshold of frame t+2 ...
+    int wide_n = 0;              // ... and the survivors of its first half
     float kc[kCache];  // this ext lane's first extension scores (-inf: none)
 #pragma unroll
     for (int k = 0; k < kCache; ++k) kc[k] = neg_inf();
@@ -773,7 +797,14 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       }
       if (lane == 0) scal[SC_NEXT_S] = c1;
       cp_async_wait_but_one();  // what was requested a frame ago has landed (visible after B1)
-      if (fused()) c2 = (t + 2 < len) ? prune_row(t + 2) : 0;
+      if (fused()) {
+        if (V <= kFusedMaxV) c2 = (t + 2 < len) ? prune_row(t + 2) : 0;
+        else if (t + 2 < len) {
+          // a wide row: the threshold and the survivors of its first half now, the rest in P3
+          wide_thr = wide_row_threshold(t + 2);
+          wide_n = wide_row_survivors(t + 2, wide_thr, 0, min(wide_half, V / 4), 0);
+        }
+      }
       if (kWide) chore_window();
     }
     if (use_bt && !is_chore) {
@@ -785,6 +816,13 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     }
     __syncthreads();  // B1
 
+    // (chore warp, wide rows) the second half of frame t+2's survivors; returns their number
+    auto finish_wide_row = [&]() -> int {
+      if (t + 2 >= len) return 0;
+      const int n = wide_row_survivors(t + 2, wide_thr, min(wide_half, V / 4), V / 4, wide_n);
+      if (lane == 0) scal[SC_KEPT] += n;
+      return n;
+    };
     // ---- P2: the cut -------------------------------------------------------------------
     // The chore warp does not scan: while the others do, it stages the log-prob table and
     // the constants of frame t+1 (and fetches the survivor count of frame t+3); it takes
@@ -1059,6 +1097,10 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
             step(q, j);
           }
         }
+      } else if (fused() && V > kFusedMaxV) {
+        // chore warp, while the others settle their candidates: the survivors of frame t+2 (by
+        // now the counts have moved up a frame: it is the frame after the next)
+        c1 = finish_wide_row();
       }
       __syncthreads();  // B3: every selected candidate is noted, the cut bin's members listed
       // P3b: one candidate per lane is written to the next beam; the chore warp meanwhile
@@ -1102,6 +1144,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       }
     } else {
       // ---- exact fallback: radix select over the integer keys ------------------------
+      if (is_chore && fused() && V > kFusedMaxV) c1 = finish_wide_row();
       auto for_each_candidate = [&](auto&& f) {
         if (is_stay) {
           for (int i = tid; i < nb; i += NS) f(score_key(st_tot[i]), i << 16);
