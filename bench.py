@@ -259,6 +259,8 @@ def run_ours(args):
         d = binding.Decoder(V, wl.blank_id, BEAM, r, B, T, device=local_rank,
                             max_trie_nodes=max(1024, BEAM * T // 2))
         d.set_profiling(True)
+        if args.no_fusion:
+            d.set_fusion(0)
         return d
 
     def barrier():
@@ -604,6 +606,8 @@ def main():
     ap.add_argument("--workload", choices=["wav2vec2", "subword"], default="wav2vec2",
                     help="default: the headline wav2vec2-shaped batch; subword: V=1024, K=32")
     ap.add_argument("--batch", type=int, default=0, help="utterances per GPU (0 = the workload's own)")
+    ap.add_argument("--no-fusion", action="store_true",
+                    help="prune with the separate kernel even where the decode kernel could do it")
     ap.add_argument("--independent", action="store_true",
                     help="N > 1: every rank draws a batch of its own instead of taking its share "
                          "of one batch of N x 64 utterances")

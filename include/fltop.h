@@ -251,7 +251,9 @@ int64_t fltop_launch_count(const fltop_handle* h);
  * out[4] the largest number of trie node ids any one utterance has used so far, out[5] probes
  * of the fingerprint table that met a different prefix with the same 20-bit tag (each was
  * told apart by the full 64 bits), out[6] frames whose selection took the slow exact path,
- * out[7] reserved (0). */
+ * out[7] non-zero if, since the handle was created, a bounded wait of the prune kernel on one of
+ * its asynchronous row copies ran out (it does not spin forever; the rows left get no
+ * survivors and the results of that call are invalid). */
 int fltop_last_call_stats(fltop_handle* h, int64_t* out);
 /* With profiling enabled every call brackets its kernels with CUDA events on the caller's
  * stream.  fltop_last_kernel_ms synchronises on those events and returns the device time
@@ -293,12 +295,16 @@ int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
  *       bounded probe walks run out, which the kernels report as FLTOP_ST_INTERNAL.
  *   FLTOP_HOOK_ROW_KERNEL      a: 1 (default) character vocabularies with beams of at most 64
  *       take the row kernel; 0: they take the general block kernel.
+ *   FLTOP_HOOK_PRUNE_STAGING   a: 1: the separate prune kernel stages rows of 1 to 4 KB through
+ *       shared memory with asynchronous bulk copies instead of holding them in registers (same
+ *       results; measured slower, kept for measurements); 0 (default): registers.
  * FLTOP_ERR_INVALID_ARG for a null handle, an unknown hook or a value out of range. */
 enum {
   FLTOP_HOOK_SURVIVOR_MASKS = 1,
   FLTOP_HOOK_PHASE_CLOCKS = 2,
   FLTOP_HOOK_TABLE_SLOTS = 3,
-  FLTOP_HOOK_ROW_KERNEL = 4
+  FLTOP_HOOK_ROW_KERNEL = 4,
+  FLTOP_HOOK_PRUNE_STAGING = 5
 };
 int fltop_set_test_hook(fltop_handle* h, int hook, void* d_buffer, int64_t a, int64_t b);
 

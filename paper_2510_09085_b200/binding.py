@@ -40,7 +40,7 @@ class fltop_config(C.Structure):
 
 FLTOP_EMISSION_F32, FLTOP_EMISSION_F16, FLTOP_EMISSION_BF16 = 0, 1, 2
 FLTOP_HOOK_SURVIVOR_MASKS, FLTOP_HOOK_PHASE_CLOCKS, FLTOP_HOOK_TABLE_SLOTS, \
-    FLTOP_HOOK_ROW_KERNEL = 1, 2, 3, 4
+    FLTOP_HOOK_ROW_KERNEL, FLTOP_HOOK_PRUNE_STAGING = 1, 2, 3, 4, 5
 EMISSION_CODES = {torch.float32: FLTOP_EMISSION_F32, torch.float16: FLTOP_EMISSION_F16,
                   torch.bfloat16: FLTOP_EMISSION_BF16}
 
@@ -335,7 +335,8 @@ class Decoder:
             raise FltopError(code, "fltop_last_call_stats")
         return {"frames": out[0], "survivors": out[1], "trie_nodes_created": out[2],
                 "live_hypotheses_sum": out[3], "max_node_ids_used": out[4],
-                "tag_clashes": out[5], "exact_select_frames": out[6]}
+                "tag_clashes": out[5], "exact_select_frames": out[6],
+                "prune_copy_timeouts": out[7]}
 
     @property
     def beam_state_bytes(self) -> int:

@@ -51,6 +51,7 @@ struct fltop_handle {
   TrieNode* nodes;
   int32_t* state;
   int32_t* stats;
+  int32_t* prune_error;   // device word: a bulk copy of the prune kernel did not complete in time
   int32_t last_B, last_T;
   bool last_fused;        // the most recent call pruned inside the decode kernel
   cudaStream_t last_stream;
@@ -69,7 +70,7 @@ struct fltop_handle {
   // instrumented launches (fltop_set_test_hook); all off by default
   uint32_t* hook_masks;
   long long* hook_clocks;
-  int32_t hook_frame0, hook_frames, hook_table_slots;
+  int32_t hook_frame0, hook_frames, hook_table_slots, hook_prune_staged;
 };
 
 namespace {
@@ -101,7 +102,7 @@ bool config_ok(const fltop_config* c) {
 }
 
 struct Layout {
-  size_t survivors, nodes, state, stats, total, beam_state;
+  size_t survivors, nodes, state, stats, flags, total, beam_state;
   size_t survivor_bytes, counts_bytes;  // the survivor region: counts, then entries
   bool survivors_inside;                // the region is part of the workspace
   int64_t frame_cap, nodes_per_utt;
@@ -134,6 +135,7 @@ Layout layout_of(const fltop_config& c) {
   if (c.max_chunk_frames > 0) off += up((size_t)c.max_batch * state_words(c.beam_width) * 4);
   l.beam_state = off;  // survivor lists (if any) + trie arenas + stream states
   l.stats = off; off += up((size_t)c.max_batch * kStatWords * sizeof(int32_t));
+  l.flags = off; off += up(sizeof(int32_t));  // device-side error word of the prune kernel
   l.total = off;
   return l;
 }
@@ -191,7 +193,9 @@ int run_decode(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t st
     h->beam_state_bytes += h->survivor_bytes;
   }
 
-  PruneParams pp;
+  PruneParams pp = {};
+  pp.error = h->prune_error;
+  pp.staged = h->hook_prune_staged;
   pp.logp = d_logp; pp.dtype = h->cfg.emission_dtype;
   pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
@@ -495,7 +499,7 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   h->warp_mode = 1;
   h->rows_mode = 1;
   h->hook_masks = nullptr; h->hook_clocks = nullptr;
-  h->hook_frame0 = h->hook_frames = h->hook_table_slots = 0;
+  h->hook_frame0 = h->hook_frames = h->hook_table_slots = h->hook_prune_staged = 0;
   h->ev[0] = h->ev[1] = h->ev[2] = nullptr;
   if (cfg->workspace) {
     h->ws = static_cast<unsigned char*>(cfg->workspace);
@@ -521,11 +525,13 @@ int fltop_create(const fltop_config* cfg, fltop_handle** out) {
   h->nodes = reinterpret_cast<TrieNode*>(h->ws + l.nodes);
   h->state = cfg->max_chunk_frames > 0 ? reinterpret_cast<int32_t*>(h->ws + l.state) : nullptr;
   h->stats = reinterpret_cast<int32_t*>(h->ws + l.stats);
+  h->prune_error = reinterpret_cast<int32_t*>(h->ws + l.flags);
   h->last_B = 0; h->last_T = 0; h->last_stream = nullptr; h->last_fused = false;
   h->frame_cap = l.frame_cap;
   h->nodes_per_utt = l.nodes_per_utt;
   h->beam_state_bytes = l.beam_state;
   e = decode_prepare(cfg->beam_width, cfg->vocab_size);
+  if (e == cudaSuccess) e = cudaMemset(h->prune_error, 0, sizeof(int32_t));
   if (e == cudaSuccess && h->state) {
     // an un-reset stream holds an empty beam rather than garbage
     e = cudaMemset(h->state, 0, (size_t)cfg->max_batch * state_words(cfg->beam_width) * 4);
@@ -584,7 +590,9 @@ int fltop_prune(fltop_handle* h, const void* d_logp, int64_t stride_b, int64_t s
   DeviceGuard g;
   cudaError_t e = g.enter(h->cfg.device);
   if (e != cudaSuccess) return cuda_fail(h, e);
-  PruneParams pp;
+  PruneParams pp = {};
+  pp.error = h->prune_error;
+  pp.staged = h->hook_prune_staged;
   pp.logp = d_logp; pp.dtype = h->cfg.emission_dtype;
   pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = h->cfg.vocab_size; pp.log_r = h->log_r;
@@ -663,6 +671,11 @@ int fltop_last_call_stats(fltop_handle* h, int64_t* out) {
     for (size_t i = 0; i < n_frames; ++i) out[1] += host[kStatWords * B + i];
   }
   delete[] host;
+  if (e == cudaSuccess) {
+    int32_t flag = 0;
+    e = cudaMemcpy(&flag, h->prune_error, sizeof(flag), cudaMemcpyDeviceToHost);
+    out[7] = flag;
+  }
   if (e != cudaSuccess) return cuda_fail(h, e);
   return FLTOP_OK;
 }
@@ -686,6 +699,10 @@ int fltop_set_test_hook(fltop_handle* h, int hook, void* d_buffer, int64_t a, in
     case FLTOP_HOOK_ROW_KERNEL:
       if (a != 0 && a != 1) return FLTOP_ERR_INVALID_ARG;
       h->rows_mode = (int32_t)a;
+      return FLTOP_OK;
+    case FLTOP_HOOK_PRUNE_STAGING:
+      if (a != 0 && a != 1) return FLTOP_ERR_INVALID_ARG;
+      h->hook_prune_staged = (int32_t)a;
       return FLTOP_OK;
     default:
       return FLTOP_ERR_INVALID_ARG;

@@ -581,6 +581,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         j1 = better ? j : j1;
         sc1 = better ? sc : sc1;
       }
+#pragma unroll 1
       for (int k = kRowCache; part + k * P < n_trows; ++k) {  // evaluated again later
         const TokLp tl = tokj[row_token(k)];
         const float sc = ((tl.tok == se.last) ? se.pb : se.tot) + tl.lp;
@@ -671,6 +672,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         count2(stot);
       } else if (is_ext && xq < nb) {
         const unsigned dw = dupw[xq];
+#pragma unroll 1
         for (int k = 0; part + k * P < n_trows; ++k) {
           const TokLp tl = tokj[row_token(k)];
           if (tl.tok >= 0 && !((dw >> tl.tok) & 1u))
@@ -848,6 +850,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
           }
         }
         // rows beyond the cache: evaluated again, a counter update per row
+#pragma unroll 1
         for (int k = kRowCache; part + k * P < n_trows; ++k) {
           const TokLp tl = tokj[row_token(k)];
           const int tok = tl.tok;
@@ -882,6 +885,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         const unsigned key_b = lane + 32 < n ? S.list_key[lane + 32] : 0u;
         const int id_b = lane + 32 < n ? S.list_id[lane + 32] : 0;
         int n_won = 0, my_m = -1, my_rank = 0;
+#pragma unroll 1
         for (int m = warp; m < n; m += NW) {
           const unsigned key = S.list_key[m];
           const int id = S.list_id[m];
@@ -920,6 +924,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
           if (tid < nb) f(score_key(stot), tid << 16);
         } else if (is_ext && xq < nb) {
           const unsigned dw = dupw[xq];
+#pragma unroll 1
           for (int k = 0; part + k * P < n_trows; ++k) {
             const TokLp tl = tokj[row_token(k)];
             const int tok = tl.tok;
@@ -944,6 +949,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         return *cnt;
       };
       unsigned kth = 0u;
+#pragma unroll 1
       for (int bit = 31; bit >= 0; --bit) {
         const unsigned trial = kth | (1u << bit);
         if (block_count([&](unsigned key, int) { return key >= trial; }) >= K) kth = trial;
@@ -952,6 +958,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
       const int need = K - n_gt;  // how many of the candidates with the K-th key fit (>= 1)
       // the need-th smallest id among them, bit by bit from the top (ids are below 2^23)
       int id_cut = 0;
+#pragma unroll 1
       for (int bit = 22; bit >= 0; --bit) {
         const int trial = id_cut | (1 << bit);
         // ids below `trial`: if fewer than `need`, the id we look for is at least `trial`

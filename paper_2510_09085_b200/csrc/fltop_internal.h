@@ -50,6 +50,8 @@ struct PruneParams {
   float log_r;
   int32_t* counts;          // [B*T]
   Survivor* entries;        // [B*T*V]
+  int32_t* error;           // one word, or-ed with 1 if a bounded wait on a bulk copy ran out; or null
+  int32_t staged;           // 1: rows that qualify go through the shared-memory ring (bulk copies)
 };
 
 struct DecodeParams {

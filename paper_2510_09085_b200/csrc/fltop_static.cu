@@ -95,7 +95,7 @@ extern "C" int fltop_decode_static(int32_t vocab_size, int32_t blank_id, int32_t
   if (e != cudaSuccess) { cudaGetLastError(); return FLTOP_ERR_CUDA; }
 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  PruneParams pp;
+  PruneParams pp = {};
   pp.logp = d_logp; pp.dtype = kEmissionF32; pp.stride_b = stride_b; pp.stride_t = stride_t; pp.lengths = d_lengths;
   pp.B = B; pp.T = T; pp.V = vocab_size;
   pp.log_r = threshold_r > 0.f ? (float)std::log((double)threshold_r)
