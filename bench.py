@@ -448,11 +448,17 @@ def run_report(args):
         B, T, V = wl.emissions.shape
         x = torch.from_numpy(wl.emissions).cuda().to(dtype)
         ln = torch.from_numpy(wl.lengths).cuda()
-        dec = binding.Decoder(V, wl.blank_id, K, r, B, T, top_n=top_n, beam_threshold=theta,
-                              merge_max=merge_max, emission_dtype=dtype)
-        dec.set_profiling(True)
-        ms, pk, dk = _time_decode(dec, x, ln, flush)
-        st = dec.last_call_stats()
+        # a trie arena of half the worst case first (peaked emissions use far less); a batch that
+        # runs out of it says so in its status words and is measured again with the worst case
+        for arena in (max(1024, K * T // 2), 0):
+            dec = binding.Decoder(V, wl.blank_id, K, r, B, T, top_n=top_n, beam_threshold=theta,
+                                  merge_max=merge_max, emission_dtype=dtype, max_trie_nodes=arena)
+            dec.set_profiling(True)
+            ms, pk, dk = _time_decode(dec, x, ln, flush)
+            st = dec.last_call_stats()
+            if int((dec.status != 0).sum()) == 0:
+                break
+            dec.close()
         assert int((dec.status != 0).sum()) == 0
         frames = int(wl.lengths.sum())
         pbytes, dbytes = _algorithmic_bytes(
@@ -467,6 +473,8 @@ def run_report(args):
                "prune_gbs": pbytes / (pk * 1e-3) / 1e9 if pk > 0 else 0.0,
                "ns_per_frame_step": 1e6 * dk / max(1, int(wl.lengths.max())),
                "beam_state_bytes": dec.beam_state_bytes,
+               "nodes_per_frame": st["max_node_ids_used"] / max(1, int(wl.lengths.max())),
+               "exact_select_frames": st["exact_select_frames"],
                "mean_survivors": st["survivors"] / max(1, st["frames"]),
                "mean_live": st["live_hypotheses_sum"] / max(1, st["frames"]), "top1_agree": agree}
         rows.append(row)
@@ -572,15 +580,16 @@ def run_report(args):
     with open(args.report, "w") as f:
         f.write(f"Measured on one B200, HBM peak {peak:.0f} GB/s ({peak_kind}); host threads {cores}.\n\n")
         f.write("| cfg | K | r | frames/s | utt/s | step ms | HBM frac (step) | prune GB/s | "
-                "ns / frame step | beam-state MB | mean survivors | mean live hyps | top-1 vs r=0 oracle |\n")
-        f.write("|---|---|---|---|---|---|---|---|---|---|---|---|---|\n")
+                "ns / frame step | beam-state MB | trie nodes / frame (max utt) | mean survivors | mean live hyps | top-1 vs r=0 oracle |\n")
+        f.write("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|\n")
         for w in rows:
             ag = "" if w["top1_agree"] is None else f"{100 * w['top1_agree']:.1f} %"
             f.write(f"| {w['workload']} | {w['K']} | {w['r']:g} | {w['frames_per_s']:.3g} | "
                     f"{w['utt_per_s']:.3g} | {w['ms']:.3f} | {100 * w['hbm_frac_step']:.3f} % | "
                     f"{(format(w['prune_gbs'], '.0f') if w['prune_gbs'] else 'in decode')} | "
                     f"{w['ns_per_frame_step']:.0f} | "
-                    f"{w['beam_state_bytes'] / 1e6:.1f} | {w['mean_survivors']:.2f} | "
+                    f"{w['beam_state_bytes'] / 1e6:.1f} | {w['nodes_per_frame']:.1f} | "
+                    f"{w['mean_survivors']:.2f} | "
                     f"{w['mean_live']:.1f} | {ag} |\n")
         f.write(f"\nStreaming (cfg 4, K={K}, r={r:g}, 1024 streams x 100 chunks of 16 frames): "
                 f"{stream_row['frames_per_s']:.3g} frames/s aggregate, chunk latency p50 "
