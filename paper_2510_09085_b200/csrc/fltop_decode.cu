@@ -139,7 +139,7 @@ enum {
   SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_MAXKEY, SC_PER_FRAME,
   // single copies
   SC_THR = 2 * SC_PER_FRAME, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_TOTAL, SC_FIRST, SC_STATUS,
-  SC_CREATED, SC_CLASHES, SC_DEAD, SC_NLIVE, SC_MADE, SC_MADE_ODD, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL, SC_KEPT,
+  SC_CREATED, SC_CLASHES, SC_EXACT, SC_DEAD, SC_NLIVE, SC_MADE, SC_MADE_ODD, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL, SC_KEPT,
   // exact fallback select
   SC_PREFIX, SC_SHIFT, SC_NEED, SC_TAKEALL, SC_DONE, SC_NBEAM_NEXT, SC_COUNT
 };
@@ -300,10 +300,16 @@ __device__ __forceinline__ void divmod_small(int e, int d, float inv_d, int& q, 
 template <int MAXT, int KMAX, int VMAX, bool BT>
 __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
-  const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
+  const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
+  const int b = p.first_wave > 0 ? utterance_by_length(p.lengths, p.B, p.T, p.first_wave,
+                                                        reinterpret_cast<int*>(smem))
+                                 : (int)blockIdx.x;
   const int K = p.K, V = p.V, blank = p.blank;
   const int KS = KMAX > 0 ? KMAX : K;  // strides of the per-entry / per-token arrays
   constexpr bool kWide = KMAX < 0;
+  // rows of more than 32 tokens pruned inside: compiled only into the instantiations that can
+  // meet them (their code costs the character-vocabulary ones a few per cent even when idle)
+  constexpr bool kWideRows = VMAX != 32;
   const int VS = VMAX > 0 ? VMAX : V;
   const Lay L = make_layout(KS, VS);
   // (a caller may shrink the table: only the test of the bounded probe walks does)
@@ -414,21 +420,23 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   // fingerprint, so a probe that meets another prefix is rejected without a second load; a
   // tag match is confirmed against the full fingerprint.  The table is at most half full, so a
   // probe sequence ends at an empty entry long before it has gone round; should it ever go
-  // round (TS probes), the walk gives up and the utterance is flagged FLTOP_ST_INTERNAL.
+  // round (back at its first slot), the walk gives up and the utterance is flagged FLTOP_ST_INTERNAL.
   auto table_insert = [&](unsigned* tab, unsigned long long h, int slot) {
     const unsigned val = (((unsigned)h & 0xfffffu) << 12) | (unsigned)slot;
-    unsigned pos = (unsigned)(h >> 40) & tmask;
-    for (int probes = 0; probes < TS; ++probes) {
+    const unsigned home = (unsigned)(h >> 40) & tmask;
+    unsigned pos = home;
+    do {
       if (atomicCAS(&tab[pos], kEmptySlot, val) == kEmptySlot) return;
       pos = (pos + 1) & tmask;
-    }
+    } while (pos != home);
     atomicOr(&scal[SC_STATUS], 16);  // FLTOP_ST_INTERNAL: the entry is not in the table
   };
   // Beam slot of the entry with fingerprint h, or -1.
   auto table_find = [&](const unsigned* tab, const Ident* ids, unsigned long long h) {
     const unsigned tag = (unsigned)h & 0xfffffu;
-    unsigned pos = (unsigned)(h >> 40) & tmask;
-    for (int probes = 0; probes < TS; ++probes) {
+    const unsigned home = (unsigned)(h >> 40) & tmask;
+    unsigned pos = home;
+    do {
       const unsigned v = tab[pos];
       if (v == kEmptySlot) return -1;
       if ((v >> 12) == tag) {
@@ -437,7 +445,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         ++tag_clashes;  // same 20-bit tag, another sequence
       }
       pos = (pos + 1) & tmask;
-    }
+    } while (pos != home);
     atomicOr(&scal[SC_STATUS], 16);  // FLTOP_ST_INTERNAL
     return -1;
   };
@@ -499,7 +507,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   // float32 rows: a word per lane; fp16 / bf16 rows: a word holds two tokens (V is even then)
   auto fetch_row = [&](int t1) {
     const int64_t at = (int64_t)b * p.stride_b + (int64_t)t1 * p.stride_t;
-    if (V > kFusedMaxV) {
+    if (kWideRows && V > kFusedMaxV) {
       // a wide row (float32, 16-byte aligned, V a multiple of four): 16 bytes per lane and turn
       const float* src = static_cast<const float*>(p.logp) + at;
       for (int c = 4 * lane; c < V; c += 128) cp_async16(raw_row(t1) + c, src + c);
@@ -560,7 +568,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     return n;
   };
   auto prune_row = [&](int t1) -> int {
-    if (V > kFusedMaxV) return prune_wide_row(t1);
+    if (kWideRows && V > kFusedMaxV) return prune_wide_row(t1);
     float v = neg_inf();
     if (p.dtype == kEmissionF32) {
       if (lane < V) v = raw_row(t1)[lane];  // the word this lane fetched itself
@@ -798,7 +806,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       if (lane == 0) scal[SC_NEXT_S] = c1;
       cp_async_wait_but_one();  // what was requested a frame ago has landed (visible after B1)
       if (fused()) {
-        if (V <= kFusedMaxV) c2 = (t + 2 < len) ? prune_row(t + 2) : 0;
+        if (!kWideRows || V <= kFusedMaxV) c2 = (t + 2 < len) ? prune_row(t + 2) : 0;
         else if (t + 2 < len) {
           // a wide row: the threshold and the survivors of its first half now, the rest in P3
           wide_thr = wide_row_threshold(t + 2);
@@ -1097,7 +1105,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
             step(q, j);
           }
         }
-      } else if (fused() && V > kFusedMaxV) {
+      } else if (kWideRows && fused() && V > kFusedMaxV) {
         // chore warp, while the others settle their candidates: the survivors of frame t+2 (by
         // now the counts have moved up a frame: it is the frame after the next)
         c1 = finish_wide_row();
@@ -1144,7 +1152,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       }
     } else {
       // ---- exact fallback: radix select over the integer keys ------------------------
-      if (is_chore && fused() && V > kFusedMaxV) c1 = finish_wide_row();
+      if (kWideRows && is_chore && fused() && V > kFusedMaxV) c1 = finish_wide_row();
       auto for_each_candidate = [&](auto&& f) {
         if (is_stay) {
           for (int i = tid; i < nb; i += NS) f(score_key(st_tot[i]), i << 16);
@@ -1160,6 +1168,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       };
       for (int i = tid; i < kPasses * kBins; i += NT) rhist[i] = 0u;
       if (tid == 0) {
+        ++scal[SC_EXACT];  // frames that needed the exact select
         scal[SC_PREFIX] = 0; scal[SC_NEED] = K; scal[SC_DONE] = 0; scal[SC_TAKEALL] = 0;
         scal[SC_SHIFT] = 0; scal[SC_NBEAM_NEXT] = K;
       }
@@ -1203,8 +1212,18 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           if (r_all || eq_rank < need) slot = total_gt + eq_rank;
           ++eq_rank;
         }
-        if (slot >= 0)
-          place_by_id(id, key, slot, (id & 0xffff) ? atomicAdd(&sc_c[SC_SLOT_E], 1) : 0);
+        if (slot >= 0) {
+          int ord = 0;
+          if (id & 0xffff) {
+            // a new prefix: numbered through one shared counter, one atomic for all lanes of the
+            // warp that are here together
+            const unsigned here = __activemask();
+            const int leader = __ffs(here) - 1;
+            if (lane == leader) ord = atomicAdd(&sc_c[SC_SLOT_E], __popc(here));
+            ord = __shfl_sync(here, ord, leader) + __popc(here & lt_mask);
+          }
+          place_by_id(id, key, slot, ord);
+        }
       });
       __syncthreads();
       if (tid == 0) scal[SC_MADE + par] = sc_c[SC_SLOT_E];
@@ -1239,7 +1258,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     if (tid == 0) {
       int32_t* o = p.stats + kStatWords * (int64_t)b;
       o[0] = len; o[1] = scal[SC_CREATED]; o[2] = live_sum - scal[SC_DEAD]; o[3] = n_nodes;
-      o[4] = scal[SC_CLASHES]; o[5] = 0;
+      o[4] = scal[SC_CLASHES]; o[5] = scal[SC_EXACT];
       o[6] = scal[SC_KEPT];  // survivors, when this kernel pruned the frames itself
     }
   }
@@ -1314,11 +1333,12 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
 
 // Layout variants: small beams over a character or a subword vocabulary get compile-time
 // array offsets, everything else the generic kernel.
-enum Variant { kCharBeam64, kSubwordBeam64, kGeneric, kWideBeam };
+enum Variant { kCharBeam64, kSubwordBeam64, kCharGeneric, kCharWideBeam, kGeneric, kWideBeam };
 constexpr int kWideBeamFrom = 257;  // measured: the wide-beam devices pay off from here
 Variant pick_variant(int K, int V) {
   if (K <= 64 && V <= 32) return kCharBeam64;
   if (K <= 64 && V <= 1024) return kSubwordBeam64;
+  if (V <= 32) return K >= kWideBeamFrom ? kCharWideBeam : kCharGeneric;
   return K >= kWideBeamFrom ? kWideBeam : kGeneric;
 }
 
@@ -1326,6 +1346,8 @@ size_t decode_smem_bytes(int K, int V) {
   switch (pick_variant(K, V)) {
     case kCharBeam64: return make_layout(64, 32).total;
     case kSubwordBeam64: return make_layout(64, 1024).total;
+    case kCharGeneric:
+    case kCharWideBeam: return make_layout(K, 32).total;
     default: return make_layout(K, V).total;
   }
 }
@@ -1344,7 +1366,10 @@ int decode_block_threads(int K, int V, bool pruning, int top_n, bool latency_bou
   }
   if (top_n > 0 && top_n < cols) cols = top_n;
   const long long stay = ((long long)K + 31) / 32 * 32;
-  long long ext = latency_bound ? (long long)K * (cols < 8 ? cols : 8) : (long long)K * cols / 3;
+  // (a character vocabulary: at most eight survivors per entry are counted; a wide one brings
+  // hundreds of survivors a frame and wants every lane it can get)
+  const long long per_entry = V > 32 ? cols : (cols < 8 ? cols : 8);
+  long long ext = latency_bound ? (long long)K * per_entry : (long long)K * cols / 3;
   ext = (ext + 31) / 32 * 32;
   if (ext < 32) ext = 32;
   long long nt = stay + ext + 32;
@@ -1352,7 +1377,7 @@ int decode_block_threads(int K, int V, bool pruning, int top_n, bool latency_bou
   // A block of at most 512 threads has 128 registers a thread instead of 64; with pruning on
   // and a beam of moderate width that is worth more than the extra lanes (measured at V = 32:
   // 3 to 12 % faster for K = 64 ... 160, slower from K = 200).
-  if (latency_bound && pruning && K <= 160 && nt > kMidBlock) nt = kMidBlock;
+  if (latency_bound && pruning && K <= 160 && V <= 32 && nt > kMidBlock) nt = kMidBlock;
   return (int)nt;
 }
 
@@ -1369,20 +1394,30 @@ cudaError_t prepare_variant(int bytes) {
   return e;
 }
 template <int KMAX, int VMAX>
-void launch_variant(const DecodeParams& p, int nt, size_t bytes, bool alone, cudaStream_t s) {
-  const bool bt = p.beam_threshold > 0.f || p.merge_max != 0;  // an option is on
+void launch_variant(const DecodeParams& p0, int nt, size_t bytes, bool alone, int sms, cudaStream_t s) {
+  const bool bt = p0.beam_threshold > 0.f || p0.merge_max != 0;  // an option is on
+  void (*kernel)(DecodeParams) = nullptr;
   if (nt <= kSmallBlock) {
-    if (bt) decode_kernel<kSmallBlock, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
-    else decode_kernel<kSmallBlock, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
+    kernel = bt ? decode_kernel<kSmallBlock, KMAX, VMAX, true> : decode_kernel<kSmallBlock, KMAX, VMAX, false>;
   } else if (nt <= kMidBlock && alone) {
     // one block per SM: it may as well have 128 registers a thread (blocks that share an SM
     // keep to 64 so that two of 512 threads fit)
-    if (bt) decode_kernel<kMidBlock, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
-    else decode_kernel<kMidBlock, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
+    kernel = bt ? decode_kernel<kMidBlock, KMAX, VMAX, true> : decode_kernel<kMidBlock, KMAX, VMAX, false>;
   } else {
-    if (bt) decode_kernel<kMaxThreads, KMAX, VMAX, true><<<p.B, nt, bytes, s>>>(p);
-    else decode_kernel<kMaxThreads, KMAX, VMAX, false><<<p.B, nt, bytes, s>>>(p);
+    kernel = bt ? decode_kernel<kMaxThreads, KMAX, VMAX, true> : decode_kernel<kMaxThreads, KMAX, VMAX, false>;
   }
+  DecodeParams p = p0;
+  if (p.first_wave > 0) {
+    // Blocks that all fit on the GPU at once: one per SM takes a long utterance, the ones that
+    // move in beside them the short ones.  More blocks than fit: longest first throughout.
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, nt, bytes) != cudaSuccess) {
+      cudaGetLastError();
+      per_sm = 1;
+    }
+    p.first_wave = (int64_t)p.B <= (int64_t)per_sm * sms ? sms : p.B;
+  }
+  kernel<<<p.B, nt, bytes, s>>>(p);
 }
 }  // namespace
 
@@ -1406,6 +1441,8 @@ cudaError_t decode_prepare(int K, int V) {
   switch (pick_variant(K, V)) {
     case kCharBeam64: return prepare_variant<64, 32>(bytes);
     case kSubwordBeam64: return prepare_variant<64, 1024>(bytes);
+    case kCharGeneric: return prepare_variant<0, 32>(bytes);
+    case kCharWideBeam: return prepare_variant<-1, 32>(bytes);
     case kWideBeam: return prepare_variant<-1, 0>(bytes);
     default: return prepare_variant<0, 0>(bytes);
   }
@@ -1420,20 +1457,29 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t s) {
   int nt = p.block_threads > 0
                ? p.block_threads
                : decode_block_threads(p.K, p.V, p.pruning != 0, p.top_n, blocks <= sms);
-  if (p.block_threads <= 0 && nt > 512 && p.pruning && blocks > sms) {
-    // more utterances than SMs: two blocks of 512 threads per SM overlap their frame chains
-    // better than one block of 1024 (measured on the subword shape, B = 256)
+  if (p.block_threads <= 0 && nt > 512 && p.pruning && blocks > 2 * sms) {
+    // many more utterances than SMs: what counts is throughput, and two blocks of 512 threads
+    // per SM overlap their frame chains better than one block of 1024.  (Up to two blocks per
+    // SM the launch lasts as long as its longest chains, which blocks of 1024 threads, started
+    // longest first, finish sooner: 4.5 against 5.1 ms on 256 utterances of 1024 tokens.)
     nt = 512;
   }
   nt = (nt + 31) / 32 * 32;
   if (nt < 96) nt = 96;  // a stay warp, an ext warp and the chore warp
   if (nt > kMaxThreads) nt = kMaxThreads;
   const size_t bytes = decode_smem_bytes(p.K, p.V);
+  DecodeParams q = p;
+  // more utterances of one batch than SMs: the blocks take them by length
+  q.first_wave = (!p.streaming && p.co_resident == 0 && p.B > sms && p.B <= kByLengthMaxB &&
+                  bytes >= (size_t)(p.B + 1) * sizeof(int))
+                     ? sms : 0;
   switch (pick_variant(p.K, p.V)) {
-    case kCharBeam64: launch_variant<64, 32>(p, nt, bytes, blocks <= sms, s); break;
-    case kSubwordBeam64: launch_variant<64, 1024>(p, nt, bytes, blocks <= sms, s); break;
-    case kWideBeam: launch_variant<-1, 0>(p, nt, bytes, blocks <= sms, s); break;
-    default: launch_variant<0, 0>(p, nt, bytes, blocks <= sms, s); break;
+    case kCharBeam64: launch_variant<64, 32>(q, nt, bytes, blocks <= sms, sms, s); break;
+    case kSubwordBeam64: launch_variant<64, 1024>(q, nt, bytes, blocks <= sms, sms, s); break;
+    case kCharGeneric: launch_variant<0, 32>(q, nt, bytes, blocks <= sms, sms, s); break;
+    case kCharWideBeam: launch_variant<-1, 32>(q, nt, bytes, blocks <= sms, sms, s); break;
+    case kWideBeam: launch_variant<-1, 0>(q, nt, bytes, blocks <= sms, sms, s); break;
+    default: launch_variant<0, 0>(q, nt, bytes, blocks <= sms, sms, s); break;
   }
   return cudaGetLastError();
 }

@@ -237,7 +237,10 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   extern __shared__ __align__(16) unsigned char smem_bytes[];
   RowsSmem<KMAX>& S = *reinterpret_cast<RowsSmem<KMAX>*>(smem_bytes);
   constexpr int kTable = RowsSmem<KMAX>::kTable;
-  const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
+  const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
+  const int b = p.first_wave > 0 ? utterance_by_length(p.lengths, p.B, p.T, p.first_wave,
+                                                        reinterpret_cast<int*>(smem_bytes))
+                                 : (int)blockIdx.x;
   const int warp = tid >> 5, NW = NT >> 5;
   const int K = p.K, V = p.V, blank = p.blank;
   const unsigned lt_mask = (1u << lane) - 1u;
@@ -1086,12 +1089,21 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
 constexpr int kRowsKmax = 64;
 
 template <int HOOKS>
-cudaError_t launch_rows_hooks(const DecodeParams& p, int nt, bool alone, cudaStream_t s) {
+cudaError_t launch_rows_hooks(const DecodeParams& p0, int nt, bool alone, int sms, cudaStream_t s) {
   const size_t bytes = sizeof(RowsSmem<kRowsKmax>);
-  if (alone && nt <= 512)
-    decode_rows_kernel<512, 1, kRowsKmax, HOOKS><<<p.B, nt, bytes, s>>>(p);
-  else
-    decode_rows_kernel<1024, 1, kRowsKmax, HOOKS><<<p.B, nt, bytes, s>>>(p);
+  void (*kernel)(DecodeParams) = (alone && nt <= 512) ? decode_rows_kernel<512, 1, kRowsKmax, HOOKS>
+                                                      : decode_rows_kernel<1024, 1, kRowsKmax, HOOKS>;
+  DecodeParams p = p0;
+  if (p.first_wave > 0) {
+    // blocks that do not all fit on the GPU at once start longest first throughout
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, nt, bytes) != cudaSuccess) {
+      cudaGetLastError();
+      per_sm = 1;
+    }
+    p.first_wave = (int64_t)p.B <= (int64_t)per_sm * sms ? sms : p.B;
+  }
+  kernel<<<p.B, nt, bytes, s>>>(p);
   return cudaGetLastError();
 }
 
@@ -1135,10 +1147,14 @@ cudaError_t launch_decode_rows(const DecodeParams& p, cudaStream_t s) {
   if (nt < 32 * (2 * nsw + 1)) nt = 32 * (2 * nsw + 1);  // stay warps, as many extension warps, the chore warp
   if (nt > kMaxThreads) nt = kMaxThreads;
   const int hooks = (p.dbg_masks ? 1 : 0) | (p.dbg_clocks ? 2 : 0);
+  DecodeParams q = p;
+  // more utterances of one batch than SMs: the blocks take them by length
+  q.first_wave = (!p.streaming && p.co_resident == 0 && p.B > sms && p.B <= kByLengthMaxB) ? sms : 0;
+  static_assert(sizeof(RowsSmem<64>) >= (kByLengthMaxB + 1) * sizeof(int), "scratch of the ranking");
   switch (hooks) {
-    case 0: return launch_rows_hooks<0>(p, nt, alone, s);
-    case 1: return launch_rows_hooks<1>(p, nt, alone, s);
-    default: return launch_rows_hooks<3>(p, nt, alone, s);
+    case 0: return launch_rows_hooks<0>(q, nt, alone, sms, s);
+    case 1: return launch_rows_hooks<1>(q, nt, alone, sms, s);
+    default: return launch_rows_hooks<3>(q, nt, alone, sms, s);
   }
 }
 

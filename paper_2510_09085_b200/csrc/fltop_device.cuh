@@ -39,6 +39,39 @@ __device__ __forceinline__ float lse2(float a, float b) {
 #endif
 }
 
+// Which utterance the calling block decodes in a launch of more blocks than SMs.  Blocks start
+// in the order of their index, so handing the utterances out by length shortens the launch:
+// the first `first_wave` blocks (one per SM) take the longest utterances, longest first, and
+// the blocks that move in beside them take the rest from the shortest upwards, so that the
+// longest frame chains share their SM for the shortest time.  Every block ranks all lengths
+// itself (length descending, index ascending: the same permutation in every block).
+// `scratch`: B + 1 ints of shared memory, free again on return.  All threads call.
+__device__ __forceinline__ int utterance_by_length(const int32_t* lengths, int B, int T,
+                                                   int first_wave, int* scratch) {
+  const int tid = threadIdx.x, NT = blockDim.x;
+  for (int i = tid; i < B; i += NT) {
+    const int l = lengths[i];
+    scratch[i] = (l < 0 || l > T) ? 0 : l;  // a bad length decodes nothing
+  }
+  __syncthreads();
+  const int blk = blockIdx.x;
+  const int want = blk < first_wave ? blk : B - 1 - (blk - first_wave);
+  for (int u = tid; u < B; u += NT) {
+    const int lu = scratch[u];
+    int rank = 0;
+    for (int v = 0; v < B; ++v) {
+      const int lv = scratch[v];
+      rank += (lv > lu || (lv == lu && v < u)) ? 1 : 0;
+    }
+    if (rank == want) scratch[B] = u;
+  }
+  __syncthreads();
+  const int b = scratch[B];
+  __syncthreads();
+  return b;
+}
+constexpr int kByLengthMaxB = 1024;  // largest batch that is handed out by length
+
 // Order-preserving map float -> uint32 (larger float = larger key).  Key 0 is
 // reserved for "not a candidate"; -inf maps there too (probability 0 is
 // dropped, as SelectTopK never keeps it).

@@ -65,6 +65,9 @@ struct DecodeParams {
   int32_t co_resident;      // utterance blocks on the GPU at the same time as this launch's,
                             // its own included (0 = just its own B): launches of one batch
                             // split over several streams size their blocks for the whole batch
+  int32_t first_wave;       // > 0: blocks take the utterances by length, the first `first_wave`
+                            // blocks the longest (a batch of more utterances than SMs, at
+                            // most 1024; see utterance_by_length)
   int32_t pruning;          // 1 when R is large enough that few tokens survive a frame
   int32_t top_n;            // survivors per frame are capped at this (0: no cap)
   float beam_threshold;     // kept prefixes score at least best - beam_threshold (<= 0: off)
