@@ -1,16 +1,19 @@
 // CTC prefix beam search over pruned frames for character vocabularies (at most 32 tokens)
-// and beams of at most 64 prefixes: the shape the paper itself decodes (Section 4: 32 tokens).
+// and beams of at most 128 prefixes: the shape the paper itself decodes (Section 4: 32 tokens).
 // Algorithm 1 with the standard CTC collapsing rule, one thread block per utterance, frames
 // walked serially, the beam in shared memory.
 //
 // A frame is a chain of dependent steps, so the design goal is the shortest chain, not
 // bandwidth.  What differs from the general block kernel (fltop_decode.cu):
 //
-//   * Every warp prunes the frame itself.  A vocabulary of at most 32 tokens is one token per
-//     lane: the row maximum is one warp reduction, the relative threshold (Algorithm 1's
-//     conditional break) one float32 add and compare, the survivors one ballot.  There is no
-//     survivor list, no token table and no per-frame constants in shared memory; the work for
-//     frame t+1 is done while the warp would otherwise wait at the last barrier of frame t.
+//   * One chore warp prepares frames ahead of their use.  A vocabulary of at most 32 tokens is
+//     one token per lane: the row maximum is one warp reduction, the relative threshold
+//     (Algorithm 1's conditional break) one float32 add and compare, the survivors one ballot.
+//     What the other warps need of a frame (log-probability by token, the surviving non-blank
+//     tokens in a row, which warp walks which of them) waits for them in a ring of four
+//     frames; the same warp alone scans the score histogram and publishes the cut.
+//   * A frame in which only blank survives changes no prefix: the beam is updated in place,
+//     and the renormalisation that was skipped is carried as a drift term.
 //   * Extension candidates are laid out as rows of "one surviving token x 32 beam entries": an
 //     extension lane owns one beam entry for the whole frame (it loads the entry once) and
 //     walks the surviving non-blank tokens that its warp is responsible for.  The work per
@@ -20,8 +23,9 @@
 //   * A candidate that lies above the cut bin of the score histogram is written into the
 //     next beam at once by the lane that owns it (slots: stays from the bottom by ballots,
 //     extensions from the top by one shared counter per warp and frame).  Only when the cut
-//     bin has to be split does a second barrier follow, after which the chore warp ranks the
-//     bin's members exactly and writes the winners in between.
+//     bin has to be split does a second barrier follow, after which all warps rank the bin's
+//     members exactly and write the winners in between; a crowded bin is first split again
+//     into 256 sub-bins.
 //   * Prefix-trie records are created only for prefixes that are new in the beam and get
 //     consecutive node ids; a frame's records leave shared memory with one bulk copy.
 //
@@ -237,6 +241,8 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   extern __shared__ __align__(16) unsigned char smem_bytes[];
   RowsSmem<KMAX>& S = *reinterpret_cast<RowsSmem<KMAX>*>(smem_bytes);
   constexpr int kTable = RowsSmem<KMAX>::kTable;
+  static_assert(KMAX == 64 || KMAX == 128, "the histogram scan takes the bits of K as a template argument");
+  constexpr int kBitsOfK = KMAX <= 64 ? 7 : 8;
   const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
   const int b = p.first_wave > 0 ? utterance_by_length(p.lengths, p.B, p.T, p.first_wave,
                                                         reinterpret_cast<int*>(smem_bytes))
@@ -334,21 +340,23 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   __syncthreads();
 
   // Table of the beam's fingerprints (open addressing, linear probing, at most one slot in
-  // sixteen taken).  Probe walks are bounded by the table size; one that goes all the way
+  // sixteen taken).  A probe walk ends at the latest back at its first slot; one that goes all the way
   // round flags the utterance FLTOP_ST_INTERNAL instead of spinning.
   auto table_insert = [&](unsigned* tab, unsigned long long h, int slot) {
     const unsigned val = (((unsigned)h & 0xfffffu) << 12) | (unsigned)slot;
-    unsigned pos = (unsigned)(h >> 40) & tmask;
-    for (int probes = 0; probes < TS; ++probes) {
+    const unsigned home = (unsigned)(h >> 40) & tmask;
+    unsigned pos = home;
+    do {
       if (atomicCAS(&tab[pos], kNoEntry, val) == kNoEntry) return;
       pos = (pos + 1) & tmask;
-    }
+    } while (pos != home);
     atomicOr(&S.bs[BS_STATUS], 16);
   };
   auto table_find = [&](const unsigned* tab, const Ident* ids, unsigned long long h) -> int {
     const unsigned tag = (unsigned)h & 0xfffffu;
-    unsigned pos = (unsigned)(h >> 40) & tmask;
-    for (int probes = 0; probes < TS; ++probes) {
+    const unsigned home = (unsigned)(h >> 40) & tmask;
+    unsigned pos = home;
+    do {
       const unsigned v = tab[pos];
       if (v == kNoEntry) return -1;
       if ((v >> 12) == tag) {
@@ -357,7 +365,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         ++tag_clashes;
       }
       pos = (pos + 1) & tmask;
-    }
+    } while (pos != home);
     atomicOr(&S.bs[BS_STATUS], 16);
     return -1;
   };
@@ -602,8 +610,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     // ---- P2: the chore warp scans the histogram; the others meanwhile empty the table that
     // the next beam's fingerprints go into
     if (is_chore) {
-      const Cut c = scan_score_histogram_ballots<7>(hist, K);
-      static_assert(KMAX <= 64, "the scan takes the bits of K as a template argument");
+      const Cut c = scan_score_histogram_ballots<kBitsOfK>(hist, K);
       if (lane == 0) {
         CutOut o;
         const bool all = c.cut_count == c.left;  // also true when there is no cut at all
@@ -684,7 +691,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
       }
       __syncthreads();
       if (is_chore) {
-        const Cut c2 = scan_score_histogram_ballots<7>(S.hist2, left);
+        const Cut c2 = scan_score_histogram_ballots<kBitsOfK>(S.hist2, left);
         if (lane == 0) {
           S.cut2[0] = c2.thr; S.cut2[1] = c2.left; S.cut2[2] = c2.cut_count;
           S.cut2[3] = c2.cut_count == c2.left ? 1 : 0;
@@ -1086,13 +1093,14 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   if (tid == 0 && p.out_status) p.out_status[b] = status;
 }
 
-constexpr int kRowsKmax = 64;
+constexpr int kRowsKmax = 128;  // widest beam; beams up to 64 have an instantiation of their own
 
-template <int HOOKS>
+template <int HOOKS, int KMAX>
 cudaError_t launch_rows_hooks(const DecodeParams& p0, int nt, bool alone, int sms, cudaStream_t s) {
-  const size_t bytes = sizeof(RowsSmem<kRowsKmax>);
-  void (*kernel)(DecodeParams) = (alone && nt <= 512) ? decode_rows_kernel<512, 1, kRowsKmax, HOOKS>
-                                                      : decode_rows_kernel<1024, 1, kRowsKmax, HOOKS>;
+  const size_t bytes = sizeof(RowsSmem<KMAX>);
+  void (*kernel)(DecodeParams) = (alone && nt <= 512) ? decode_rows_kernel<512, 1, KMAX, HOOKS>
+                                                      : decode_rows_kernel<1024, 1, KMAX, HOOKS>;
+  static_assert(sizeof(RowsSmem<KMAX>) <= 48 * 1024, "fits without the opt-in attribute");
   DecodeParams p = p0;
   if (p.first_wave > 0) {
     // blocks that do not all fit on the GPU at once start longest first throughout
@@ -1130,6 +1138,9 @@ int decode_rows_threads(const DecodeParams& p, bool alone) {
   const int cap = ((alone ? 16 : 8) - 1 - nsw) / nsw;
   if (alone && p.pruning && nsw > 1 && P > 4) P = 4;
   if (P > cap) P = cap;
+  // beams above 96 without pruning: four warps per block of entries (21 warps) beat the cap's two
+  // (K = 100, r = 0: 4.8 against 6.1 ms)
+  if (alone && !p.pruning && nsw >= 4 && rows >= 8) P = 4;
   if (P < 1) P = 1;
   return 32 * (nsw + 1 + nsw * P);
 }
@@ -1151,10 +1162,17 @@ cudaError_t launch_decode_rows(const DecodeParams& p, cudaStream_t s) {
   // more utterances of one batch than SMs: the blocks take them by length
   q.first_wave = (!p.streaming && p.co_resident == 0 && p.B > sms && p.B <= kByLengthMaxB) ? sms : 0;
   static_assert(sizeof(RowsSmem<64>) >= (kByLengthMaxB + 1) * sizeof(int), "scratch of the ranking");
+  if (p.K <= 64) {
+    switch (hooks) {
+      case 0: return launch_rows_hooks<0, 64>(q, nt, alone, sms, s);
+      case 1: return launch_rows_hooks<1, 64>(q, nt, alone, sms, s);
+      default: return launch_rows_hooks<3, 64>(q, nt, alone, sms, s);
+    }
+  }
   switch (hooks) {
-    case 0: return launch_rows_hooks<0>(q, nt, alone, sms, s);
-    case 1: return launch_rows_hooks<1>(q, nt, alone, sms, s);
-    default: return launch_rows_hooks<3>(q, nt, alone, sms, s);
+    case 0: return launch_rows_hooks<0, 128>(q, nt, alone, sms, s);
+    case 1: return launch_rows_hooks<1, 128>(q, nt, alone, sms, s);
+    default: return launch_rows_hooks<3, 128>(q, nt, alone, sms, s);
   }
 }
 

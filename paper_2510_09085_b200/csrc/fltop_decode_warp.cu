@@ -130,24 +130,26 @@ __global__ void __launch_bounds__(32 * kWarpsPerBlock) decode_warp_kernel(Decode
     if (lane < n) {
       const unsigned long long h = e_print;
       const unsigned val = (((unsigned)h & 0xfffffu) << 12) | (unsigned)lane;
-      unsigned pos = (unsigned)(h >> 40) & (kWarpTab - 1);
+      const unsigned home = (unsigned)(h >> 40) & (kWarpTab - 1);
+      unsigned pos = home;
       bool in = false;
-      for (int probes = 0; probes < kWarpTab && !in; ++probes) {
+      do {  // (ends at the latest back at its first slot)
         in = atomicCAS(&S.tab[pos], kFree, val) == kFree;
         pos = (pos + 1) & (kWarpTab - 1);
-      }
+      } while (!in && pos != home);
       if (!in) status |= 16;  // FLTOP_ST_INTERNAL (cannot happen: 32 entries, 128 slots)
     }
   };
   auto table_find = [&](const BeamCopy& c, unsigned long long h) -> int {
     const unsigned tag = (unsigned)h & 0xfffffu;
-    unsigned pos = (unsigned)(h >> 40) & (kWarpTab - 1);
-    for (int probes = 0; probes < kWarpTab; ++probes) {
+    const unsigned home = (unsigned)(h >> 40) & (kWarpTab - 1);
+    unsigned pos = home;
+    do {
       const unsigned v = S.tab[pos];
       if (v == kFree) return -1;
       if ((v >> 12) == tag && c.print[v & 0xfffu] == h) return (int)(v & 0xfffu);
       pos = (pos + 1) & (kWarpTab - 1);
-    }
+    } while (pos != home);
     return -1;
   };
   auto clear_frame_scratch = [&]() {

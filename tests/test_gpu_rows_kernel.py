@@ -39,7 +39,9 @@ def _run(em, ln, K, r, rows=True, nt=0, **kw):
 @pytest.mark.parametrize("V,K,r,top_n", [(32, 50, 1e-3, 0), (32, 50, 0.0, 0), (32, 64, 1e-2, 0),
                                          (32, 8, 0.01, 0), (32, 33, 0.3, 0), (32, 20, 7e-3, 4),
                                          (32, 16, 0.5, 1), (5, 12, 0.05, 2), (2, 4, 0.0, 0),
-                                         (17, 1, 0.0, 0), (3, 64, 0.0, 0), (31, 40, 1e-4, 0)])
+                                         (17, 1, 0.0, 0), (3, 64, 0.0, 0), (31, 40, 1e-4, 0),
+                                         (32, 65, 1e-3, 0), (32, 100, 0.0, 0), (32, 128, 1e-2, 0),
+                                         (32, 97, 7e-3, 4), (6, 128, 0.0, 0)])
 def test_row_kernel_matches_oracle_and_block_kernel(V, K, r, top_n):
     B = 9
     em, ln = W.make_small(7300 + V + K, B, 70, 70, V)
@@ -188,9 +190,9 @@ def test_row_kernel_more_utterances_than_sms():
     d.close()
 
 
-@pytest.mark.parametrize("C", [1, 3, 16])
-def test_row_kernel_streaming_equals_one_shot(C):
-    V, K, r, B = 32, 40, 1e-2, 6
+@pytest.mark.parametrize("C,K", [(1, 40), (3, 40), (16, 40), (5, 100)])
+def test_row_kernel_streaming_equals_one_shot(C, K):
+    V, r, B = 32, 1e-2, 6
     em, ln = W.make_small(7800 + C, B, 5, 70, V)
     T = em.shape[1]
     x = _dev(em)
