@@ -89,9 +89,9 @@ struct __align__(8) Where {
 };
 
 // per-frame scalars, one set per frame parity
-enum { FS_SLOT_E = 0, FS_WIN_E, FS_LISTN, FS_NSTAY, FS_COUNT = 8 };  // (the first two: one 8-byte load)
+enum { FS_SLOT_E = 0, FS_WIN_E, FS_LISTN, FS_NSTAY, FS_MAXKEY, FS_COUNT = 8 };  // (the first two: one 8-byte load)
 // block scalars
-enum { BS_STATUS = 0, BS_CLASHES, BS_NLIVE, BS_EXACT, BS_CNT0, BS_CNT1, BS_CNT2, BS_COUNT = 16 };
+enum { BS_STATUS = 0, BS_CLASHES, BS_NLIVE, BS_EXACT, BS_CNT0, BS_CNT1, BS_CNT2, BS_DEAD, BS_COUNT = 16 };
 // What the scan of the score histogram found, as the scanning warp publishes it: everything
 // the other warps need, ready to use.
 struct __align__(16) CutOut {
@@ -236,7 +236,10 @@ __device__ __forceinline__ int nth_set_bit(unsigned m, int n) {
 
 // HOOKS bit 0: the survivor mask of every frame is written out (tests); bit 1: the clock at
 // every phase boundary is recorded for block 0 (profiling).  Shipped launches use HOOKS = 0.
-template <int MAXT, int MINB, int KMAX, int HOOKS>
+// BT: SelectTopK's beam_threshold is on - the exact best score of every frame is tracked, and a
+// candidate that wins a slot but scores below best - beam_threshold is written as a dead slot
+// (probability 0, no identity, not in the table): it yields no candidates and no hypothesis.
+template <int MAXT, int MINB, int KMAX, int HOOKS, bool BT>
 __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p) {
   extern __shared__ __align__(16) unsigned char smem_bytes[];
   RowsSmem<KMAX>& S = *reinterpret_cast<RowsSmem<KMAX>*>(smem_bytes);
@@ -252,6 +255,9 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   const unsigned lt_mask = (1u << lane) - 1u;
   const int TS = p.table_slots > 0 ? min(p.table_slots, kTable) : kTable;
   const unsigned tmask = (unsigned)TS - 1u;
+  // masses of one prefix are summed, or (merge_max) the larger one is taken: Algorithm 1's
+  // literal score' = score + logit, a prefix scores as its best alignment
+  const bool use_max = p.merge_max != 0;
 
   // ---- roles ---------------------------------------------------------------------------
   const int nsw = (K + 31) >> 5;            // stay warps: one lane per beam entry
@@ -494,6 +500,10 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         chore_window();
         if (t + 2 < len) prepare_layout(t + 2);
       }
+      if (BT && is_stay) {  // dead slots stay dead and are not counted as held prefixes
+        const unsigned dead = __ballot_sync(kFull, tid < nb && S.hot[cur][tid].tot == neg_inf());
+        if (lane == 0 && dead) atomicAdd(&S.bs[BS_DEAD], __popc(dead));
+      }
       drift += head.lp_blank;
       pend_bytes = 0u;
       live_sum += nb;
@@ -532,6 +542,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     float kc[kRowCache];
 #pragma unroll
     for (int k = 0; k < kRowCache; ++k) kc[k] = neg_inf();
+    float far_max = neg_inf();               // (BT) best score among the rows beyond the cache
     float sc1 = neg_inf(), sc2 = neg_inf();  // best and second-best cached score of this lane
     int j1 = 0, tok1 = 0;                    // position and token of the best
     unsigned long long hp = 0ull, h1 = 0ull; // fingerprints of the entry and of the best candidate
@@ -566,7 +577,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
             }
           }
         }
-        stot = lse3(npb, own, dup);
+        stot = use_max ? fmaxf(npb, fmaxf(own, dup)) : lse3(npb, own, dup);
         if (stot != neg_inf()) atomicAdd(&hist[score_bin(stot)], 1u);
         s_own = own;
         s_dup = dup;
@@ -597,6 +608,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         const TokLp tl = tokj[row_token(k)];
         const float sc = ((tl.tok == se.last) ? se.pb : se.tot) + tl.lp;
         if (sc != neg_inf()) atomicAdd(&hist[score_bin(sc)], 1u);
+        if (BT) far_max = fmaxf(far_max, sc);
       }
       tok1 = tokj[j1].tok;
       if (sc1 != neg_inf()) h1 = child_print(hp, tok1);
@@ -625,6 +637,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         o.empty = c.total == 0 ? 1 : 0;
         o.thr = c.thr;
         S.cut = o;
+
       }
     } else {
       if (is_stay) {
@@ -634,7 +647,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         // what a stay candidate needs only if it is kept, and the other stay warps'
         // candidates: fetched and worked out while the scan runs
         if (tid < nb) {
-          npnb = lse2(s_own, s_dup);
+          npnb = use_max ? fmaxf(s_own, s_dup) : lse2(s_own, s_dup);
           swh = wh_c[tid];
         }
 #pragma unroll
@@ -651,6 +664,22 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     int n_listed = cut.n_listed, left = cut.left;
     const int nbn = cut.nbn;
     const bool arena_ok = n_nodes + ((K + 1) & ~1) <= nodes_cap;
+    // (BT) SelectTopK's beam_threshold: kept scores reach the frame's exact best minus the
+    // threshold.  No score lies above the reference edge by more than log 3 (a stay candidate
+    // sums three masses that are each below it), so when even the lower edge of the cut bin
+    // is within the threshold of that bound nothing can be dropped and the exact best is not
+    // needed; otherwise the block reduces it (one more barrier).
+    float floor_sc = neg_inf();
+    if (BT && f_lo < best + 2.f - p.beam_threshold) {  // block-uniform
+      if (is_stay || has_rows) {
+        // (an absorbed extension never beats the stay candidate it went into)
+        const unsigned key = __reduce_max_sync(kFull, score_key(is_stay ? stot : fmaxf(sc1, far_max)));
+        if (lane == 0 && key) atomicMax(reinterpret_cast<unsigned*>(&fs[FS_MAXKEY]), key);
+      }
+      __syncthreads();
+      const unsigned mk = (unsigned)fs[FS_MAXKEY];
+      if (mk) floor_sc = key_score(mk) - p.beam_threshold;
+    }
 
     // A crowded cut bin (more members than the pairwise ranking takes) is binned once more:
     // an inner bin into 256 sub-bins over its quarter nat, the last bin - everything more
@@ -716,8 +745,17 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     }
 
     // writing candidates into the next beam
+    auto place_dead = [&](int slot) {
+      Hot e;
+      e.last = -1; e.pb = e.pnb = e.tot = neg_inf();
+      hn[slot] = e;
+      id_n[slot] = Ident{0ull, 0ull};
+      wh_n[slot] = Where{0, 0};
+      atomicAdd(&S.bs[BS_DEAD], 1);
+    };
     auto place_stay_from = [&](int q, float pb_q, float pnb_q, float tot_q, int slot) {
       if ((unsigned)slot >= (unsigned)K) return;  // only reachable with NaN scores
+      if (BT && tot_q < floor_sc) return place_dead(slot);
       Hot e;
       e.last = hc[q].last; e.pb = pb_q - best; e.pnb = pnb_q - best; e.tot = tot_q - best;
       hn[slot] = e;
@@ -731,12 +769,13 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
     auto place_new = [&](unsigned long long hp_q, Where w_q, int tok, unsigned long long h,
                          float sc, int slot, int ord) {
       if ((unsigned)slot >= (unsigned)K || (unsigned)ord >= (unsigned)K) return;
+      nst[ord] = TrieNode{w_q.node, tok};  // (also for a dead slot: the frame's records are one run)
+      if (BT && sc < floor_sc) return place_dead(slot);
       Hot e;
       e.last = tok; e.pb = neg_inf(); e.pnb = sc - best; e.tot = sc - best;
       hn[slot] = e;
       id_n[slot] = Ident{h, hp_q};
       wh_n[slot] = Where{arena_ok ? n_nodes + ord : 0, w_q.len + 1};
-      nst[ord] = TrieNode{w_q.node, tok};
       table_insert(tab_n, h, slot);
     };
     auto place_ext = [&](int q, int tok, float sc, int slot, int ord) {
@@ -791,7 +830,9 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
         if (tid == 0) fs[FS_NSTAY] = total_sel;
         if (kl == 2) {
           const int slot = before + __popc(m_own & lt_mask);
-          if ((unsigned)slot < (unsigned)K) {
+          if (BT && (unsigned)slot < (unsigned)K && stot < floor_sc) {
+            place_dead(slot);
+          } else if ((unsigned)slot < (unsigned)K) {
             Hot e;
             e.last = se.last; e.pb = npb - best; e.pnb = npnb - best; e.tot = stot - best;
             hn[slot] = e;
@@ -1023,7 +1064,7 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
   status |= S.bs[BS_STATUS];
   if (p.stats && tid == 0) {
     int32_t* o = p.stats + kStatWords * (int64_t)b;
-    o[0] = len; o[1] = created_sum; o[2] = live_sum; o[3] = n_nodes;
+    o[0] = len; o[1] = created_sum; o[2] = live_sum - S.bs[BS_DEAD]; o[3] = n_nodes;
     o[4] = S.bs[BS_CLASHES]; o[5] = S.bs[BS_EXACT];
   }
 
@@ -1095,11 +1136,11 @@ __global__ void __launch_bounds__(MAXT, MINB) decode_rows_kernel(DecodeParams p)
 
 constexpr int kRowsKmax = 128;  // widest beam; beams up to 64 have an instantiation of their own
 
-template <int HOOKS, int KMAX>
+template <int HOOKS, int KMAX, bool BT = false>
 cudaError_t launch_rows_hooks(const DecodeParams& p0, int nt, bool alone, int sms, cudaStream_t s) {
   const size_t bytes = sizeof(RowsSmem<KMAX>);
-  void (*kernel)(DecodeParams) = (alone && nt <= 512) ? decode_rows_kernel<512, 1, KMAX, HOOKS>
-                                                      : decode_rows_kernel<1024, 1, KMAX, HOOKS>;
+  void (*kernel)(DecodeParams) = (alone && nt <= 512) ? decode_rows_kernel<512, 1, KMAX, HOOKS, BT>
+                                                      : decode_rows_kernel<1024, 1, KMAX, HOOKS, BT>;
   static_assert(sizeof(RowsSmem<KMAX>) <= 48 * 1024, "fits without the opt-in attribute");
   DecodeParams p = p0;
   if (p.first_wave > 0) {
@@ -1118,8 +1159,10 @@ cudaError_t launch_rows_hooks(const DecodeParams& p0, int nt, bool alone, int sm
 }  // namespace
 
 bool decode_rows_eligible(const DecodeParams& p) {
-  return p.K <= kRowsKmax && p.V <= kRowsMaxV && p.logp != nullptr && !(p.beam_threshold > 0.f) &&
-         p.merge_max == 0;
+  // (the instrumented instantiations exist without beam_threshold only)
+  const bool hooked = p.dbg_masks != nullptr || p.dbg_clocks != nullptr;
+  return p.K <= kRowsKmax && p.V <= kRowsMaxV && p.logp != nullptr &&
+         !(p.beam_threshold > 0.f && hooked);
 }
 
 // Threads per block: the stay warps, the chore warp, and for every block of 32 beam entries P
@@ -1162,6 +1205,10 @@ cudaError_t launch_decode_rows(const DecodeParams& p, cudaStream_t s) {
   // more utterances of one batch than SMs: the blocks take them by length
   q.first_wave = (!p.streaming && p.co_resident == 0 && p.B > sms && p.B <= kByLengthMaxB) ? sms : 0;
   static_assert(sizeof(RowsSmem<64>) >= (kByLengthMaxB + 1) * sizeof(int), "scratch of the ranking");
+  if (p.beam_threshold > 0.f) {
+    return p.K <= 64 ? launch_rows_hooks<0, 64, true>(q, nt, alone, sms, s)
+                     : launch_rows_hooks<0, 128, true>(q, nt, alone, sms, s);
+  }
   if (p.K <= 64) {
     switch (hooks) {
       case 0: return launch_rows_hooks<0, 64>(q, nt, alone, sms, s);
