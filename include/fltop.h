@@ -71,8 +71,10 @@ enum {
 
 typedef struct {
   int32_t vocab_size;     /* V, 2 <= V <= 8192; V and K together must fit one SM's shared
-                             memory (about 48 V + 130 K bytes <= 227 KB: V = 4096 with small
-                             beams, K = 1500 at V = 32), else fltop_create refuses */
+                             memory (about 48 V + 130 K bytes <= 227 KB, plus 16 bytes a token
+                             for 32 < V <= 1024, whose rows the decode block keeps four frames
+                             of: V = 4096 with small beams, K = 1500 at V = 32), else
+                             fltop_create refuses */
   int32_t blank_id;       /* 0 <= blank_id < V */
   int32_t beam_width;     /* K = beam_size of Algorithm 1, 1 <= K <= 2048 */
   float threshold_r;      /* R of Algorithm 1 in the probability domain, 0 <= R <= 1;
@@ -239,7 +241,7 @@ const char* fltop_status_string(int code);
 int fltop_last_cuda_error(const fltop_handle* h);
 /* Bytes of beam state the handle holds now: prefix trie arenas, stream states and - once a
  * call has needed them - the survivor lists of the separate prune kernel (vocabularies above
- * 32 tokens get them at fltop_create; narrower ones only if a call cannot prune inside the
+ * 1024 tokens get them at fltop_create; narrower ones only if a call cannot prune inside the
  * decode kernel, see fltop_set_fusion, and then by a device allocation of the library's own
  * even when the handle lives in a caller's workspace). */
 size_t fltop_beam_state_bytes(const fltop_handle* h);
@@ -264,14 +266,18 @@ int fltop_set_profiling(fltop_handle* h, int enable);
  * the library choose from K, V and R).  A tuning knob: results do not depend on it. */
 int fltop_set_block_threads(fltop_handle* h, int32_t threads);
 /* Where the frames are pruned (Algorithm 1, the top-N stage and the conditional break).
- * mode 1 (the default): inside the decode kernel whenever vocab_size <= 32 - each utterance
- * block fetches its own emission rows and no survivor list goes through device memory;
- * wider vocabularies take the separate prune kernel.  mode 0: always the separate kernel.
- * Results do not depend on it.  FLTOP_ERR_INVALID_ARG for a null handle or another mode. */
+ * mode 1 (the default): inside the decode kernel whenever it can - each utterance block (or
+ * warp) fetches its own emission rows and no survivor list goes through device memory.  It
+ * can for vocab_size <= 32 with any element type, and for vocab_size <= 1024 with float32
+ * emissions whose rows start on 16-byte boundaries (vocab_size and both strides multiples of
+ * four, d_logp 16-byte aligned) and no top_n cap.  Everything else takes the separate prune
+ * kernel, which writes [B,T,V] survivor pairs that the decode kernel reads back.  mode 0:
+ * always the separate kernel.  The survivors are the same bit for bit either way, the
+ * hypotheses the same up to the order of exactly tied ones.  FLTOP_ERR_INVALID_ARG for a null handle or another mode. */
 int fltop_set_fusion(fltop_handle* h, int mode);
 /* Which decode kernel serves narrow problems (beam_width <= 32, vocab_size <= 32, pruning
- * inside the kernel, no beam_threshold, no merge_max, no block size set).  The library has two:
- * one thread block per utterance, and one warp per utterance with several utterances to a block.
+ * inside the kernel, no beam_threshold, no merge_max, no block size set).  The library has two
+ * kinds: one thread block per utterance, and one warp per utterance with several utterances to a block.
  * A warp alone is slower on its utterance but an SM runs many more of them side by side.
  * mode 1 (the default): the warp kernel when a call brings at least eight utterances or streams
  * per SM; mode 0: never; mode 2: whenever the problem is narrow enough.  Results are the same up
@@ -282,7 +288,8 @@ int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
 /* Instrumented launches, for tests and profiling; everything is off on a new handle and no
  * ordinary launch pays for it.  The paper has no counterpart.
  *   FLTOP_HOOK_SURVIVOR_MASKS  d_buffer: DEVICE uint32 [B*T] of the next calls (NULL = off).
- *       A decode kernel that prunes the frames itself (vocab_size <= 32) writes the survivor
+ *       A decode kernel that prunes the frames of a vocabulary of at most 32 tokens itself
+ *       writes the survivor
  *       set of frame (b,t) - bit c set iff token c survives Algorithm 1's top-N stage and
  *       conditional break - to d_buffer[b*T + t]; frames past the length are left untouched.
  *   FLTOP_HOOK_PHASE_CLOCKS    d_buffer: DEVICE int64 [b][32][8] (NULL = off): for frames
@@ -293,8 +300,8 @@ int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
  *   FLTOP_HOOK_TABLE_SLOTS     a: 0 (off) or a power of two: the shared-memory table of prefix
  *       fingerprints is cut down to that many slots.  With fewer slots than beam entries its
  *       bounded probe walks run out, which the kernels report as FLTOP_ST_INTERNAL.
- *   FLTOP_HOOK_ROW_KERNEL      a: 1 (default) character vocabularies with beams of at most 64
- *       take the row kernel; 0: they take the general block kernel.
+ *   FLTOP_HOOK_ROW_KERNEL      a: 1 (default) vocabularies of at most 32 tokens with beams of at
+ *       most 128 take the row kernel; 0: they take the general block kernel.
  *   FLTOP_HOOK_PRUNE_STAGING   a: 1: the separate prune kernel stages rows of 1 to 4 KB through
  *       shared memory with asynchronous bulk copies instead of holding them in registers (same
  *       results; measured slower, kept for measurements); 0 (default): registers.
