@@ -60,10 +60,11 @@ def test_wav2vec2_batch_pruned(wav2vec2):
     assert _compare_sampled(wav2vec2, 50, 1e-3, list(range(64)), frac=0.0) == 0
 
 
-def test_wav2vec2_batch_unpruned_sampled(wav2vec2):
-    order = np.argsort(wav2vec2.lengths)
-    sample = [int(order[i]) for i in (0, 9, 20, 31, 40, 52, 63)]
-    _compare_sampled(wav2vec2, 50, 0.0, sample)
+def test_wav2vec2_batch_unpruned(wav2vec2):
+    # the benchmark's second leg, r = 0: every utterance
+    n = _compare_sampled(wav2vec2, 50, 0.0, list(range(64)), frac=0.0)
+    print(f"wav2vec2 r=0: {n} unmatched hypotheses of {64 * 50}")
+    assert n == 0
 
 
 def test_wav2vec2_survivors_bit_exact(wav2vec2):
@@ -140,22 +141,26 @@ def test_survivor_masks_inside_the_decode_kernels_bit_exact(wav2vec2):
 
 @pytest.mark.parametrize("K", W.SWEEP_BEAMS)
 @pytest.mark.parametrize("r", W.SWEEP_THRESHOLDS)
-def test_sweep_cells_sampled(wav2vec2, K, r):
-    # every cell of the beam / threshold sweep, two utterances each (the shortest two for the
-    # widest beams, where the oracle is slow; a short and a middling one otherwise)
+def test_sweep_cells(wav2vec2, K, r):
+    # every cell of the beam / threshold sweep: all 64 utterances; for the widest beams, where
+    # the oracle is slow, the shorter half.  Not one hypothesis outside the oracle's beam.
     order = np.argsort(wav2vec2.lengths)
-    sample = [int(order[0]), int(order[1])] if K >= 500 else [int(order[0]), int(order[24])]
-    _compare_sampled(wav2vec2, K, r, sample)
+    sample = [int(order[i]) for i in range(32 if K >= 500 else 64)]
+    n = _compare_sampled(wav2vec2, K, r, sample, frac=0.0)
+    print(f"sweep K={K} r={r}: {n} unmatched hypotheses of {len(sample) * K}")
+    assert n == 0
 
 
-def test_subword_batch_sampled():
+def test_subword_batch():
     wl = W.workload_subword()
     order = np.argsort(wl.lengths)
     d = gpu_decode(wl.emissions, wl.lengths, wl.blank_id, 32, 1e-3)
-    sample = [int(order[i]) for i in (0, 1, 2, 40, 80, 128, 170, 200, 230, 255)]
-    _compare_sampled(wl, 32, 1e-3, sample, d=d)
+    sample = [int(order[i]) for i in range(0, 256, 2)]  # every other utterance by length
+    n = _compare_sampled(wl, 32, 1e-3, sample, frac=0.0, d=d)
+    print(f"subword r=1e-3: {n} unmatched hypotheses of {len(sample) * 32}")
+    assert n == 0
     d.close()
-    _compare_sampled(wl, 32, 0.0, [int(order[0]), int(order[3])])
+    _compare_sampled(wl, 32, 0.0, [int(order[i]) for i in (0, 3, 9, 20, 35, 50, 70, 90)])
     # survivors bit exact on the same input
     B, T, V = wl.emissions.shape
     d = _binding().Decoder(V, 0, 2, 1e-3, B, T)
