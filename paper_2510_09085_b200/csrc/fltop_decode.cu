@@ -136,7 +136,7 @@ struct __align__(16) FrameInfo {
 
 enum {
   // one copy per frame parity
-  SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_MAXKEY, SC_PER_FRAME,
+  SC_LISTN = 0, SC_SLOT, SC_SLOT_E, SC_MAXKEY, SC_WIN_E, SC_PER_FRAME,
   // single copies
   SC_THR = 2 * SC_PER_FRAME, SC_LEFT, SC_CUT_COUNT, SC_CUT_BASE, SC_TOTAL, SC_FIRST, SC_STATUS,
   SC_CREATED, SC_CLASHES, SC_EXACT, SC_DEAD, SC_NLIVE, SC_MADE, SC_MADE_ODD, SC_NEXT_S, SC_NEXT_BJ, SC_NEXT_BL, SC_KEPT,
@@ -1002,7 +1002,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     const int n_listed = refined ? (take_all2 ? 0 : sub_count) : (take_all ? 0 : cut.cut_count);
     const int n_winners = refined ? sub_left : cut.left;
 
-    if (take_all || use_list || (refined && n_listed <= kListCap)) {
+    const bool fast_select = take_all || use_list || (refined && n_listed <= kListCap);  // block-uniform
+    if (fast_select) {
       // P3a: every candidate above the cut bin takes a beam slot and is noted there; stays
       // fill the beam from slot 0 upwards, extensions from the last slot downwards.
       auto list_add = [&](unsigned key, int id) {
@@ -1126,29 +1127,42 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
           const int slot = nbn - 1 - x;
           if (slot >= 0) place_by_id(sel_id[slot], sel_key[slot], slot, x);
         }
-      } else {
-        // (the extensions among the winners are numbered after those placed above)
+      }
+      // The members of the cut bin are ranked by (score, candidate id) and the best n_winners
+      // go to the slots between the stays and the extensions.  All warps share the work: a warp
+      // takes every NW-th member and counts, with one ballot per 32 members, how many beat it;
+      // then one lane per winner writes it.  (The extensions among the winners are numbered
+      // after those placed above.)
+      if (n_listed > 0) {  // block-uniform
+        const int n = min(n_listed, kListCap);
         const int n_ext = min(sc_c[SC_SLOT_E], K);
-        int won_ext = 0;
-        for (int base = 0; base < n_listed; base += 32) {
-          const int li = base + lane;
-          unsigned key = 0u;
-          int id = 0, rank = 0x7fffffff;
-          if (li < n_listed) {
-            key = list_key[li];
-            id = list_id[li];
-            rank = 0;
-            for (int j = 0; j < n_listed; ++j) {
-              const unsigned kj = list_key[j];
-              rank += (kj > key || (kj == key && list_id[j] < id)) ? 1 : 0;
-            }
+        const unsigned key_a = lane < n ? list_key[lane] : 0u;
+        const int id_a = lane < n ? list_id[lane] : 0;
+        const unsigned key_b = lane + 32 < n ? list_key[lane + 32] : 0u;
+        const int id_b = lane + 32 < n ? list_id[lane + 32] : 0;
+        int n_won = 0, my_m = -1, my_rank = 0;
+        for (int m = warp; m < n; m += NW) {
+          const unsigned key = list_key[m];
+          const int id = list_id[m];
+          int rank = __popc(__ballot_sync(kFull, lane < n && (key_a > key || (key_a == key && id_a < id))));
+          if (n > 32)
+            rank += __popc(__ballot_sync(
+                kFull, lane + 32 < n && (key_b > key || (key_b == key && id_b < id))));
+          if (rank < n_winners) {
+            if (lane == n_won) { my_m = m; my_rank = rank; }
+            ++n_won;
           }
-          const bool won = rank < n_winners;
-          const unsigned mx = __ballot_sync(kFull, won && (id & 0xffff) != 0);
-          if (won) place_by_id(id, key, n_stay + rank, n_ext + won_ext + __popc(mx & lt_mask));
-          won_ext += __popc(mx);
         }
-        if (lane == 0) scal[SC_MADE + par] = n_ext + won_ext;  // new prefixes of this frame
+        if (n_won) {  // warp-uniform; lane i writes the i-th winner this warp found
+          const bool mine = my_m >= 0;
+          const int id = mine ? list_id[my_m] : 0;
+          const unsigned mx = __ballot_sync(kFull, mine && (id & 0xffff) != 0);
+          int base = 0;
+          if (lane == 0 && mx) base = atomicAdd(&sc_c[SC_WIN_E], __popc(mx));
+          base = __shfl_sync(kFull, base, 0);
+          if (mine)
+            place_by_id(id, list_key[my_m], n_stay + my_rank, n_ext + base + __popc(mx & lt_mask));
+        }
       }
     } else {
       // ---- exact fallback: radix select over the integer keys ------------------------
@@ -1233,7 +1247,8 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     __syncthreads();  // B4: the next beam and its hash table are complete
 
     // (chore warp) what the next frame has to write out
-    const int made = min(scal[SC_MADE + par], K);  // new prefixes: consecutive node ids
+    // new prefixes of the frame (they have consecutive node ids)
+    const int made = min(fast_select ? min(sc_c[SC_SLOT_E], K) + sc_c[SC_WIN_E] : scal[SC_MADE + par], K);
     pend_at = n_nodes;
     pend_bytes = (arena_ok && made > 0) ? (unsigned)(((made + 1) & ~1) * sizeof(TrieNode)) : 0u;
     if (!arena_ok && made > 0) status |= 2;  // FLTOP_ST_ARENA_FULL
