@@ -307,6 +307,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   const int K = p.K, V = p.V, blank = p.blank;
   const int KS = KMAX > 0 ? KMAX : K;  // strides of the per-entry / per-token arrays
   constexpr bool kWide = KMAX < 0;
+  constexpr int kBitsOfK = KMAX == 64 ? 7 : 12;  // bits of the widest beam (the histogram scan counts over them)
   // rows of more than 32 tokens pruned inside: compiled only into the instantiations that can
   // meet them (their code costs the character-vocabulary ones a few per cent even when idle)
   constexpr bool kWideRows = VMAX != 32;
@@ -856,7 +857,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     Cut cut;
     if (warp_scans) {
       if (!is_chore) {
-        cut = scan_score_histogram(hist, K);
+        cut = scan_score_histogram_ballots<kBitsOfK>(hist, K);
         if (warp == 0) {
           if (lane == 0) publish_cut(cut);
           __threadfence_block();
@@ -871,7 +872,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       // large blocks: warp 0 scans, all the others stage the tables of frame t+1 together
       const int S_next = scal[SC_NEXT_S];
       if (warp == 0) {
-        cut = scan_score_histogram(hist, K);
+        cut = scan_score_histogram_ballots<kBitsOfK>(hist, K);
         if (lane == 0) publish_cut(cut);
       } else {
         if (t + 1 < len) stage_tables(t + 1, fi.S, S_next, tid - 32, NT - 32);

@@ -105,84 +105,6 @@ struct __align__(16) CutOut {
   int thr;         // the cut bin
 };
 
-// One warp turns the score histogram into the cut (all lanes get the result).  Lane l owns bins
-// [8l, 8l + 8).  The prefix counts over lanes come from ballots over the bits of the lanes'
-// counts (clamped to K, which leaves the place where the running count reaches K unchanged):
-// independent instructions instead of a chain of shuffles.  KBITS: bits of K.
-template <int KBITS>
-__device__ __forceinline__ Cut scan_score_histogram_ballots(const unsigned* hist, int K) {
-  const int lane = threadIdx.x & 31;
-  const unsigned le_mask = 0xffffffffu >> (31 - lane);  // lanes up to and including this one
-  {
-    // Fast path: the K-th best score lies in the first 32 bins (within 8 nats of the
-    // reference), one bin per lane.  This is the usual case: the reference follows the best.
-    const int v = (int)hist[lane];
-    const int vc = min(v, K);
-    int inc1 = 0;
-#pragma unroll
-    for (int bit = 0; bit < KBITS; ++bit)
-      inc1 += __popc(__ballot_sync(kFull, (vc >> bit) & 1) & le_mask) << bit;
-    const unsigned reach1 = __ballot_sync(kFull, inc1 >= K);
-    if (reach1) {
-      const int owner = __ffs(reach1) - 1;
-      const unsigned any1 = __ballot_sync(kFull, v != 0);
-      Cut r;
-      r.first = (__ffs(any1) - 1) >> 3;
-      r.total = K;  // at least
-      r.thr = owner;
-      r.cut_base = __shfl_sync(kFull, inc1 - vc, owner);
-      r.cut_count = __shfl_sync(kFull, v, owner);
-      r.left = K - r.cut_base;
-      return r;
-    }
-  }
-  const uint4 lo4 = reinterpret_cast<const uint4*>(hist)[2 * lane];
-  const uint4 hi4 = reinterpret_cast<const uint4*>(hist)[2 * lane + 1];
-  int pre[kBinsPerLane];  // inclusive prefix counts inside the lane
-  pre[0] = (int)lo4.x; pre[1] = (int)(lo4.x + lo4.y);
-  pre[2] = pre[1] + (int)lo4.z; pre[3] = pre[1] + (int)(lo4.z + lo4.w);
-  const int h01 = (int)(hi4.x + hi4.y), h23 = (int)(hi4.z + hi4.w);
-  pre[4] = pre[3] + (int)hi4.x; pre[5] = pre[3] + h01;
-  pre[6] = pre[5] + (int)hi4.z; pre[7] = pre[3] + (h01 + h23);
-  const int c = pre[7];
-  const int cc = min(c, K);
-  int inc = 0;  // inclusive prefix of the clamped counts over lanes
-#pragma unroll
-  for (int bit = 0; bit < KBITS; ++bit)
-    inc += __popc(__ballot_sync(kFull, (cc >> bit) & 1) & le_mask) << bit;
-  const unsigned any = __ballot_sync(kFull, c != 0);
-  const unsigned reach = __ballot_sync(kFull, inc >= K);
-  Cut r;
-  r.first = any ? __ffs(any) - 1 : 0;
-  if (!reach) {  // fewer than K candidates: every one is kept (no count was clamped)
-    r.total = __shfl_sync(kFull, inc, 31);
-    r.thr = kFastBins; r.left = 0; r.cut_count = 0; r.cut_base = r.total;
-    return r;
-  }
-  // The lane in which the running count reaches K: before it no count was clamped, so its
-  // own prefix counts are exact.
-  const int owner = __ffs(reach) - 1;
-  const int before = inc - cc;
-  int n_below = 0, base = before, at_cut = 0x7fffffff;
-#pragma unroll
-  for (int i = 0; i < kBinsPerLane; ++i) {
-    const int v = before + pre[i];
-    const bool below = v < K;
-    n_below += below ? 1 : 0;
-    base = below ? max(base, v) : base;
-    at_cut = below ? at_cut : min(at_cut, v);
-  }
-  // thr in the top bits, the bin's population and the count above it below
-  const unsigned packed = ((unsigned)n_below << 28) | ((unsigned)(at_cut - base) << 12) | (unsigned)base;
-  const unsigned got = __shfl_sync(kFull, packed, owner);
-  r.total = K;  // at least
-  r.thr = owner * kBinsPerLane + (int)(got >> 28);
-  r.cut_count = (int)((got >> 12) & 0xffffu);
-  r.cut_base = (int)(got & 0xfffu);
-  r.left = K - r.cut_base;
-  return r;
-}
-
 // What every warp has to know about a frame, prepared once by the chore warp a frame ahead.
 struct __align__(8) TokLp {
   int tok;     // -1: no such survivor
