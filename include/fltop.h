@@ -296,7 +296,10 @@ int fltop_last_kernel_ms(fltop_handle* h, float* out_ms);
  *       a <= t < a + b of utterance 0 the row kernel records the SM clock of every warp at its
  *       eight phase boundaries (frame start, end of evaluation, after the first barrier, after
  *       the histogram scan, end of placement, after the list barrier, before and after the
- *       last barrier).
+ *       last barrier).  The general block kernel (without beam_threshold / merge_max) records
+ *       its own eight marks for the utterance of block 0: frame start, candidates evaluated,
+ *       past the first barrier, cut known, candidates settled, at the second barrier (large
+ *       blocks), next beam written, past the last barrier.
  *   FLTOP_HOOK_TABLE_SLOTS     a: 0 (off) or a power of two: the shared-memory table of prefix
  *       fingerprints is cut down to that many slots.  With fewer slots than beam entries its
  *       bounded probe walks run out, which the kernels report as FLTOP_ST_INTERNAL.

@@ -297,7 +297,9 @@ __device__ __forceinline__ void divmod_small(int e, int d, float inv_d, int& q, 
 // candidate anew every frame).
 // BT: an option of Algorithm 1 beyond N and R is on - beam_threshold (the exact best score of
 // every frame is tracked) and / or merging by max instead of log-sum.
-template <int MAXT, int KMAX, int VMAX, bool BT>
+// CLK: every warp of block 0 records the SM clock at its phase boundaries (profiling; only the
+// instantiations for blocks of up to 1024 threads without options exist with it).
+template <int MAXT, int KMAX, int VMAX, bool BT, bool CLK = false>
 __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
@@ -646,6 +648,14 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
   unsigned pend_bytes = 0u;
   for (int t = 0; t < len; ++t) {
     const int par = t & 1, nxt = cur ^ 1;
+    // marks: 0 frame start, 1 candidates evaluated, 2 past B1, 3 the cut is known, 4 candidates
+    // settled (before B3), 5 at B2 (large blocks), 6 next beam written (before B4), 7 past B4
+    auto clock_mark = [&](int i) {
+      if (CLK && blockIdx.x == 0 && lane == 0 && p.dbg_clocks && t >= p.dbg_frame0 &&
+          t < p.dbg_frame0 + p.dbg_frames)
+        p.dbg_clocks[((int64_t)(t - p.dbg_frame0) * 32 + warp) * 8 + i] = clock64();
+    };
+    clock_mark(0);
     const Survivor* const sv = svbuf(t);
     const float* const lpv = lpvbuf(t);
     const Hot* const hc = hot_base + cur * KS;
@@ -823,7 +833,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
       if (lane == 0 && my_max != neg_inf())
         atomicMax(reinterpret_cast<unsigned*>(&sc_c[SC_MAXKEY]), score_key(my_max));
     }
+    clock_mark(1);
     __syncthreads();  // B1
+    clock_mark(2);
 
     // (chore warp, wide rows) the second half of frame t+2's survivors; returns their number
     auto finish_wide_row = [&]() -> int {
@@ -882,6 +894,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         for (int i = tid - 32; i < TS / 4; i += NT - 32) tb_n[i] = ones;
         if (!kWide && is_chore) chore_window();
       }
+      clock_mark(5);
       __syncthreads();  // B2 (large blocks only)
       read_cut(cut);
       if (is_chore) {
@@ -890,6 +903,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         c0 = c1; c1 = c2; c2 = c3;
       }
     }
+    clock_mark(3);
     // new zero of the relative scores: the upper edge of the first non-empty group of bins
     const float best = -(float)(cut.first * kBinsPerLane) * (1.f / kBinsPerNat);
     const bool take_all = cut.cut_count == cut.left;  // also true when there is no cut at all
@@ -1112,6 +1126,7 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
         // now the counts have moved up a frame: it is the frame after the next)
         c1 = finish_wide_row();
       }
+      clock_mark(4);
       __syncthreads();  // B3: every selected candidate is noted, the cut bin's members listed
       // P3b: one candidate per lane is written to the next beam; the chore warp meanwhile
       // ranks the members of the cut bin exactly (score, then candidate id) and writes the
@@ -1245,7 +1260,9 @@ __global__ void __launch_bounds__(MAXT) decode_kernel(DecodeParams p) {
     }
     if (cut.total == 0) status |= 8;  // FLTOP_ST_EMPTY_BEAM
     offset += (double)best;
+    clock_mark(6);
     __syncthreads();  // B4: the next beam and its hash table are complete
+    clock_mark(7);
 
     // (chore warp) what the next frame has to write out
     // new prefixes of the frame (they have consecutive node ids)
@@ -1407,6 +1424,8 @@ cudaError_t prepare_variant(int bytes) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kSmallBlock, KMAX, VMAX, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMidBlock, KMAX, VMAX, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX, true>, attr, bytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_kernel<kMaxThreads, KMAX, VMAX, false, true>, attr, bytes);
   return e;
 }
 template <int KMAX, int VMAX>
@@ -1422,6 +1441,8 @@ void launch_variant(const DecodeParams& p0, int nt, size_t bytes, bool alone, in
   } else {
     kernel = bt ? decode_kernel<kMaxThreads, KMAX, VMAX, true> : decode_kernel<kMaxThreads, KMAX, VMAX, false>;
   }
+  // (phase clocks: the instrumented instantiation, whatever the block size)
+  if (p0.dbg_clocks && !bt) kernel = decode_kernel<kMaxThreads, KMAX, VMAX, false, true>;
   DecodeParams p = p0;
   if (p.first_wave > 0) {
     // Blocks that all fit on the GPU at once: one per SM takes a long utterance, the ones that

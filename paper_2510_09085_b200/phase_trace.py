@@ -1,6 +1,8 @@
-"""Phase-by-phase clock trace of the row kernel's frame loop.
+"""Phase-by-phase clock trace of a decode kernel's frame loop.
 
     python -m paper_2510_09085_b200.phase_trace [--beam 50] [--r 1e-3] [--frames 400]
+    python -m paper_2510_09085_b200.phase_trace --workload subword --beam 32     (the block kernel)
+    python -m paper_2510_09085_b200.phase_trace --beam 500                       (the block kernel)
 
 Decodes the wav2vec2-shaped batch (64 utterances, 32 tokens) with the instrumented launch of
 the row kernel (``fltop_set_test_hook``, FLTOP_HOOK_PHASE_CLOCKS): every warp of utterance 0's
@@ -10,6 +12,10 @@ the previous phase to the moment the slowest warp leaves this one), which warp w
 the same split by kind of frame.  The instrumented launch is slower than the ordinary one (a
 clock read and a global store per mark), so proportions, not absolute cycle counts, are what
 this is for; frames in which only blank survives have no phases and are only counted.
+
+Vocabularies above 32 tokens and beams above 128 are decoded by the general block kernel, whose
+instrumented instantiation marks its own phases (evaluate, cut, settle, write, tail); the block
+traced is block 0, which in a batch of more utterances than SMs decodes the longest utterance.
 """
 from __future__ import annotations
 
@@ -31,10 +37,14 @@ def main():
     ap.add_argument("--first", type=int, default=50)
     ap.add_argument("--frames", type=int, default=400)
     ap.add_argument("--threads", type=int, default=0)
+    ap.add_argument("--workload", choices=["wav2vec2", "subword"], default="wav2vec2")
     args = ap.parse_args()
-    wl = W.workload_wav2vec2()
+    wl = W.workload_wav2vec2() if args.workload == "wav2vec2" else W.workload_subword()
     B, T, V = wl.emissions.shape
-    nf = min(args.frames, int(wl.lengths[0]) - args.first)
+    block_kernel = V > 32 or args.beam > 128
+    # (block 0 of a batch of more utterances than SMs takes the longest one)
+    traced_utt = int(np.argmax(wl.lengths)) if B > 148 else 0
+    nf = min(args.frames, int(wl.lengths[traced_utt]) - args.first)
     x = torch.from_numpy(wl.emissions).cuda()
     ln = torch.from_numpy(wl.lengths).cuda()
     d = bd.Decoder(V, wl.blank_id, args.beam, args.r, B, T)
@@ -46,6 +56,10 @@ def main():
     d.decode(x, ln)
     torch.cuda.synchronize()
     c = buf.cpu().numpy()
+    if block_kernel:
+        trace_block_kernel(c, args, nf)
+        d.close()
+        return
     nw = int((c[:, :24, 0] > 0).any(axis=0).sum())
     traced = [f for f in range(nf) if c[f, :nw, 0].min() > 0]
     print(f"K={args.beam} r={args.r:g}: {nw} warps, frames {args.first}..{args.first + nf - 1} of "
@@ -89,6 +103,50 @@ def main():
     for k in ("few survivors", "many survivors (>= 16)", "cut bin ranked"):
         show(kinds == k, k)
     d.close()
+
+
+BLOCK_PHASES = ["evaluate (P1)", "cut (P2)", "settle (P3a)", "write (P3b)", "tail to next frame"]
+
+
+def trace_block_kernel(c, args, nf):
+    """Marks of the block kernel: 0 frame start, 1 candidates evaluated, 2 past B1, 3 cut known,
+    4 candidates settled (before B3), 5 at B2 (large blocks), 6 next beam written, 7 past B4."""
+    nw = int((c[:, :, 0] > 0).any(axis=0).sum())
+    rows, last, skipped = [], [], 0
+    for f in range(nf - 1):
+        w = c[f, :nw]
+        if w[:, 4].max() == 0:      # the exact select took this frame: no settle mark
+            skipped += 1
+            continue
+        start, p1, p2 = w[:, 0].min(), w[:, 1].max(), w[:, 3].max()
+        p3, p4, nx = w[:, 4].max(), w[:, 6].max(), c[f + 1, :nw, 0].min()
+        rows.append([p1 - start, p2 - p1, p3 - p2, p4 - p3, nx - p4])
+        last.append([int(w[:, 1].argmax()), int(w[:, 3].argmax()), int(w[:, 4].argmax()),
+                     int(w[:, 6].argmax())])
+    rows, last = np.array(rows, dtype=np.float64), np.array(last)
+    print(f"{args.workload} K={args.beam} r={args.r:g}: block kernel, {nw} warps, frames "
+          f"{args.first}..{args.first + nf - 1} of the utterance of block 0; {skipped} frames went "
+          f"through the exact select (not shown)")
+    print(f"\n{len(rows)} frames, {rows.sum(axis=1).mean():.0f} cycles a frame on average")
+    role = lambda w: "chore" if w == nw - 1 else ("warp 0" if w == 0 else "others")
+    for j, name in enumerate(BLOCK_PHASES):
+        who = ""
+        if j < 4:
+            roles = [role(int(w)) for w in last[:, j]]
+            who = "  last: " + ", ".join(f"{k} {roles.count(k) * 100 // len(roles)} %"
+                                         for k in ("warp 0", "others", "chore") if k in roles)
+        print(f"  {name:20s} mean {rows[:, j].mean():7.0f}  max {rows[:, j].max():7.0f}{who}")
+    ok = c[: nf - 1, :nw, 4].max(axis=1) > 0
+    w = c[: nf - 1, :nw][ok]
+    rel = lambda mark, base: (w[:, :, mark] - base)
+    s0 = w[:, :, 0].min(axis=1, keepdims=True)
+    b1 = w[:, :, 2].max(axis=1, keepdims=True)
+    ck = w[:, :, 3].max(axis=1, keepdims=True)
+    for label, m, base in (("evaluated, after the frame's start", 1, s0), ("at B2, after B1", 5, b1),
+                           ("settled, after the cut", 4, ck)):
+        r = rel(m, base)
+        print(f"  {label:36s} warp 0 {r[:, 0].mean():6.0f}   others mean {r[:, 1:nw - 1].mean():6.0f} "
+              f"max {r[:, 1:nw - 1].max(axis=1).mean():6.0f}   chore {r[:, nw - 1].mean():6.0f}")
 
 
 if __name__ == "__main__":
