@@ -142,6 +142,9 @@ def trace_block_kernel(c, args, nf):
     s0 = w[:, :, 0].min(axis=1, keepdims=True)
     b1 = w[:, :, 2].max(axis=1, keepdims=True)
     ck = w[:, :, 3].max(axis=1, keepdims=True)
+    own = w[:, :, 4] - w[:, :, 3]   # each warp's own time from knowing the cut to having settled
+    print(f"  {'settled, after the warp itself knew the cut':36s} warp 0 {own[:, 0].mean():6.0f}   others mean "
+          f"{own[:, 1:nw - 1].mean():6.0f} max {own[:, 1:nw - 1].max(axis=1).mean():6.0f}   chore {own[:, nw - 1].mean():6.0f}")
     for label, m, base in (("evaluated, after the frame's start", 1, s0), ("at B2, after B1", 5, b1),
                            ("settled, after the cut", 4, ck)):
         r = rel(m, base)
